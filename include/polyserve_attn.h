@@ -1,0 +1,256 @@
+/*
+ * polyserve_attn.h -- C ABI of the mixed-batch paged-KV attention library.
+ *
+ * One serving-instance iteration batches every running decode request with a
+ * dynamically sized chunk of prefill tokens (paper section 2.4, chunked
+ * prefill; section 4.7, dynamic chunking).  The attention step of that
+ * iteration is Softmax(Q K^T / sqrt(d)) V over the K, V of all previous tokens
+ * (section 2.1), per request, with the K, V held in a paged cache addressed
+ * through a block table.  The scheduler predicts iteration time from a profiled
+ * table keyed by token batch size and KV-cache size (section 4.5); the sweep
+ * entry point below emits that table for the attention step.
+ *
+ * Notation: request r has prior[r] >= 0 tokens attended in earlier iterations
+ * and q_len[r] >= 1 new tokens; kv_len[r] = prior[r] + q_len[r].  New token i
+ * of request r attends keys 0 .. prior[r] + i (itself included).  Q head h
+ * reads KV head h / (n_q_heads / n_kv_heads).  All kv_len[r] tokens' K and V,
+ * the new ones included, are in the cache before ps_attn_run is called.
+ *
+ * Conventions
+ *   - every function returns a ps_status; nothing throws across the boundary;
+ *   - "host" / "dev" in a parameter name says where the pointer must live;
+ *   - streams are cudaStream_t passed as void* (NULL = the default stream);
+ *   - the caller owns Q, out, block table, workspace and (optionally) the pool
+ *     memory; the library owns the handles it returns;
+ *   - no entry point synchronises the device unless its comment says so;
+ *   - the library targets sm_100a only and has no CPU path: without a usable
+ *     device every launching call returns PS_ERR_CUDA.
+ */
+#ifndef POLYSERVE_ATTN_H_
+#define POLYSERVE_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PS_OK = 0,
+    PS_ERR_INVALID = 1,     /* bad argument (null pointer, negative length, q_len < 1, ...) */
+    PS_ERR_OOM = 2,         /* host or device allocation failed */
+    PS_ERR_CUDA = 3,        /* a CUDA runtime call failed; see ps_last_error() */
+    PS_ERR_UNSUPPORTED = 4, /* shape outside what the kernels handle */
+    PS_ERR_WORKSPACE = 5,   /* workspace smaller than the plan requires */
+    PS_ERR_BOUNDS = 6,      /* device saw a page id outside the pool */
+    PS_ERR_TIMEOUT = 7      /* a bounded device-side wait expired */
+} ps_status;
+
+/* Attention geometry.  Supported: head_dim in {64, 128}, page_size == 16,
+ * n_q_heads a multiple of n_kv_heads, dtype == 0 (bf16 in, fp32 accumulate,
+ * bf16 out). */
+typedef struct {
+    int32_t n_q_heads;
+    int32_t n_kv_heads;
+    int32_t head_dim;
+    int32_t page_size;
+    int32_t dtype;
+} ps_shape;
+
+typedef struct ps_kv ps_kv;     /* paged K/V pool                       */
+typedef struct ps_plan ps_plan; /* work partition of one batch of lengths */
+
+/* Planner options; a NULL pointer or a zero field selects the default. */
+typedef struct {
+    int32_t decode_segment_tokens;  /* KV tokens per decode work item (multiple of page_size); 0 = auto */
+    int32_t prefill_segment_tokens; /* KV tokens per prefill work item (multiple of 128); 0 = auto */
+    int32_t num_sms;                /* SM count to balance for; 0 = ask the current device */
+} ps_plan_opts;
+
+/* ------------------------------------------------------------------------ */
+/* Paged KV pool (the paged cache and block table of section 6.1's serving    */
+/* engines; cache population of section 2.1).                                 */
+/* ------------------------------------------------------------------------ */
+
+/* Bytes a pool of num_pages pages occupies. */
+ps_status ps_kv_bytes(const ps_shape *shape, int64_t num_pages, size_t *bytes_out);
+
+/*
+ * Create a pool of num_pages pages of page_size tokens.  If dev_mem is NULL
+ * the library allocates the pool with cudaMalloc and frees it in ps_kv_free;
+ * otherwise dev_mem (device memory, 1024-byte aligned, dev_bytes >=
+ * ps_kv_bytes()) stays owned by the caller and must outlive the handle.  The
+ * physical layout inside a page is private to the library: fill the pool with
+ * ps_kv_write and read it back with ps_kv_gather.  Pool contents are not
+ * initialised.  Which pages a sequence uses is the caller's decision, passed
+ * in as the block table.
+ */
+ps_status ps_kv_alloc(const ps_shape *shape, int64_t num_pages, void *dev_mem, size_t dev_bytes, ps_kv **out);
+ps_status ps_kv_free(ps_kv *kv);
+
+/*
+ * Scatter the K, V of new tokens into their pages (section 2.1: each pass
+ * populates the KV cache).  k_new_dev / v_new_dev: bf16 [T, n_kv_heads,
+ * head_dim], T = sum q_len, requests in batch order, tokens in order.  Token i
+ * of request r goes to logical position prior_host[r] + i, i.e. page
+ * block_table_dev[r * max_pages + pos / page_size], slot pos % page_size.
+ * Asynchronous on `stream`; lengths are read before the call returns.
+ * Errors: PS_ERR_INVALID for null pointers, q_len < 1, prior < 0 or a position
+ * beyond max_pages * page_size; page ids outside the pool are skipped on the
+ * device and reported by ps_kv_status.
+ */
+ps_status ps_kv_write(ps_kv *kv, const void *k_new_dev, const void *v_new_dev, const int32_t *block_table_dev,
+                      int32_t max_pages, const int32_t *prior_host, const int32_t *q_len_host, int32_t n,
+                      void *stream);
+
+/*
+ * Copy logical tokens [0, len) of one sequence out of the pool, bit for bit,
+ * into contiguous bf16 [len, n_kv_heads, head_dim] buffers (either may be
+ * NULL).  block_table_row_dev: that sequence's page ids (device).  Asynchronous.
+ */
+ps_status ps_kv_gather(const ps_kv *kv, const int32_t *block_table_row_dev, int32_t len, void *k_out_dev,
+                       void *v_out_dev, void *stream);
+
+/* Synchronises `stream`, then returns PS_OK or PS_ERR_BOUNDS for the pool's
+ * write/gather kernels since the last call, and clears the flag. */
+ps_status ps_kv_status(ps_kv *kv, void *stream);
+
+/* ------------------------------------------------------------------------ */
+/* Work partition (host only).                                                */
+/* ------------------------------------------------------------------------ */
+
+/*
+ * Partition one batch into work items.  Rows with q_len == 1 are decode rows
+ * (memory-bound KV streaming, section 2.2); rows with q_len > 1 are prefill
+ * chunks (dense contraction, section 3.4).  Long contexts are cut into KV
+ * segments whose partial results a merge kernel combines.  Host arrays
+ * prior_host / q_len_host have n entries and are read before the call returns.
+ * max_pages_per_seq is the row stride of the block table later given to
+ * ps_attn_run; kv_len[r] must not exceed max_pages_per_seq * page_size.
+ *
+ * *plan_inout == NULL creates a plan; otherwise the existing plan is rebuilt
+ * in place, reusing its pinned staging memory (the call first waits until the
+ * plan's last ps_attn_run has finished reading that memory).  Running the
+ * device is not needed: the only CUDA calls are pinned-memory management and,
+ * if opts->num_sms == 0, a device-attribute query.
+ * *workspace_bytes_out: device bytes ps_attn_run needs for this plan.
+ * Errors: PS_ERR_INVALID (n < 1, q_len < 1, prior < 0, kv_len too long),
+ * PS_ERR_UNSUPPORTED (shape), PS_ERR_OOM.
+ */
+ps_status ps_attn_plan(const ps_shape *shape, const int32_t *prior_host, const int32_t *q_len_host, int32_t n,
+                       int32_t max_pages_per_seq, const ps_plan_opts *opts, ps_plan **plan_inout,
+                       size_t *workspace_bytes_out);
+ps_status ps_plan_free(ps_plan *plan);
+
+/* Counts describing a plan, for tests and reports. */
+typedef struct {
+    int32_t n_decode_items;
+    int32_t n_prefill_items;
+    int32_t n_merge_rows;      /* (token, q head) outputs that need the merge kernel */
+    int32_t decode_segment_tokens;
+    int32_t prefill_segment_tokens;
+    int64_t n_partial_slots;   /* fp32 partial rows held in the workspace */
+    int64_t total_q_tokens;
+    int32_t n_launches;        /* kernels one ps_attn_run launches for this plan */
+} ps_plan_info;
+ps_status ps_plan_get_info(const ps_plan *plan, ps_plan_info *info_out);
+
+/*
+ * Copy the plan's work items to host arrays for inspection (tests check that
+ * the items cover every (row, q head, visible key) exactly once).  Each item is
+ * 8 int32: {request, kv_head, key_begin, key_end, q_token, n_tokens,
+ * partial_slot, first_position}.  q_token is the packed index of the item's
+ * first q token, n_tokens how many consecutive q tokens it covers (1 for
+ * decode), partial_slot is -1 when the item writes final output, and
+ * first_position = prior + index of its first token in the chunk.  Either
+ * output may be NULL; capacities are in items.
+ */
+ps_status ps_plan_get_items(const ps_plan *plan, int32_t *decode_items_out, int64_t decode_capacity,
+                            int32_t *prefill_items_out, int64_t prefill_capacity);
+
+/* ------------------------------------------------------------------------ */
+/* Attention for one iteration.                                               */
+/* ------------------------------------------------------------------------ */
+
+/*
+ * out[t, h, :] = sum_j softmax_j(q[t, h, :] . K[j, g, :] / sqrt(d)) V[j, g, :]
+ * over the keys the token may see (section 2.1).  q_dev / out_dev: bf16
+ * [T, n_q_heads, head_dim] packed as for ps_kv_write; lse_out_dev: optional
+ * fp32 [T, n_q_heads], natural-log sum of exponentials of the scaled scores
+ * (NULL to skip).  block_table_dev: int32 [n, max_pages_per_seq] page ids;
+ * entries past a sequence's last page are never read.  workspace_dev: device
+ * memory (256-byte aligned) of at least the plan's workspace bytes; its
+ * contents need no initialisation and are scratch.  Asynchronous on `stream`:
+ * one small host-to-device copy of the work list, then the decode, prefill
+ * and merge kernels.  Two runs of the same plan must not overlap on the device.
+ * Returns host-detectable errors only (PS_ERR_INVALID, PS_ERR_WORKSPACE,
+ * PS_ERR_CUDA); errors seen on the device are read with ps_plan_status.
+ */
+ps_status ps_attn_run(ps_plan *plan, const ps_kv *kv, const void *q_dev, const int32_t *block_table_dev,
+                      void *out_dev, float *lse_out_dev, void *workspace_dev, size_t workspace_bytes,
+                      void *stream);
+
+/* Synchronises `stream`, then reports what the plan's last run saw on the
+ * device: PS_OK, PS_ERR_BOUNDS (a page id outside the pool; that page was
+ * skipped) or PS_ERR_TIMEOUT (a bounded wait expired; output is invalid). */
+ps_status ps_plan_status(ps_plan *plan, void *stream);
+
+/* ------------------------------------------------------------------------ */
+/* Latency-table sweep (section 4.5: a profiled map from batch size and KV    */
+/* cache size to execution time, which the scheduler consults).               */
+/* ------------------------------------------------------------------------ */
+
+typedef struct {
+    const int32_t *chunk_sizes;   int32_t n_chunk_sizes;   /* prefill chunk tokens; 0 = no chunk */
+    const int32_t *decode_counts; int32_t n_decode_counts; /* decode rows per batch */
+    const int32_t *mean_ctxs;     int32_t n_mean_ctxs;     /* mean context length m */
+    int32_t seeds_per_cell;       /* independent length draws per cell */
+    int32_t warmup;               /* untimed runs per draw (>= 1) */
+    int32_t iters;                /* timed runs per draw (>= 1) */
+    uint64_t seed_base;           /* draw s of cell c uses seed seed_base + seeds_per_cell * c + s */
+} ps_grid_spec;
+
+typedef struct {
+    int32_t chunk, n_decode, mean_ctx, seed_index;
+    uint64_t seed;
+    int32_t token_batch;      /* chunk + n_decode: the table's "batch size" key */
+    int32_t prefill_prior;    /* prior context drawn for the chunk */
+    int64_t kv_tokens;        /* sum of kv_len: the table's "KV cache size" key */
+    double decode_bytes;      /* kv_len * bytes of K+V per token, summed over decode rows */
+    double prefill_flops;     /* 4 d Hq (c prior + c (c + 1) / 2) */
+    float latency_us;         /* median over iters of one ps_attn_run, CUDA events */
+    float latency_min_us;
+    float latency_max_us;
+    float plan_us;            /* host time of ps_attn_plan for this draw */
+} ps_grid_row;
+
+/*
+ * Time ps_attn_run over chunk_sizes x decode_counts x mean_ctxs x seeds.
+ * Per draw: decode contexts (kv_len) are integers uniform on [m/2, 3m/2], the
+ * chunk's prior context is one more draw of that law; pages are assigned by a
+ * seeded permutation of a pool with 25 % spare pages.  Lengths come from
+ * SplitMix64 streams keyed by the draw's seed, so a caller can regenerate
+ * them.  K, V and Q hold bounded pseudo-random bf16 values; small batches
+ * rotate over several copies of the pool so that no run finds its KV in L2.
+ * The library allocates and frees all device memory it needs (largest cell x
+ * rotation) and synchronises the device; `stream` is used for the timed runs.
+ * rows (host, capacity max_rows) receives one row per draw in sweep order
+ * (chunk-major, then decode count, then mean context, then seed);
+ * *n_rows_out is the count written.  If csv_path is not NULL the rows are also
+ * written there as CSV with a header line.
+ * Errors: PS_ERR_INVALID (null/empty spec, max_rows too small),
+ * PS_ERR_UNSUPPORTED, PS_ERR_OOM, PS_ERR_CUDA; a device-side error of any run
+ * aborts the sweep with that status.
+ */
+ps_status ps_profile_grid(const ps_shape *shape, const ps_grid_spec *spec, ps_grid_row *rows, int64_t max_rows,
+                          int64_t *n_rows_out, const char *csv_path, void *stream);
+
+/* Thread-local text of the last error returned on this thread ("" if none). */
+const char *ps_last_error(void);
+const char *ps_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POLYSERVE_ATTN_H_ */

@@ -1,0 +1,241 @@
+// Internal declarations shared by the library's translation units: error
+// plumbing, the KV pool layout, the device work-list records and thin wrappers
+// over the PTX the kernels use (mbarrier, bulk async copy, ldmatrix, mma).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/polyserve_attn.h"
+
+namespace ps {
+
+// ---------------------------------------------------------------------------
+// errors
+// ---------------------------------------------------------------------------
+ps_status fail(ps_status code, const char* fmt, ...);
+void clear_error();
+
+#define PS_CUDA_TRY(expr)                                                                     \
+    do {                                                                                      \
+        cudaError_t e__ = (expr);                                                             \
+        if (e__ != cudaSuccess)                                                               \
+            return ps::fail(PS_ERR_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), \
+                            __FILE__, __LINE__);                                              \
+    } while (0)
+
+ps_status check_shape(const ps_shape* s);
+
+// ---------------------------------------------------------------------------
+// KV pool layout
+//
+// A page holds kPage = 16 tokens.  For one (page, kv head) the pool stores a
+// K block followed by a V block, each 16 * d bf16:
+//     pool + ((page * Hkv + g) * 2 + kv) * (16 * d * 2 bytes)
+// A block is d / 64 "halves" of [16 tokens][64 elements = 128 bytes]; inside a
+// half the eight 16-byte units of token row t are stored at unit index
+// u ^ (t & 7).  This is the 128-byte-swizzle pattern that both ldmatrix
+// (conflict-free 8x8 fetches) and the tcgen05 shared-memory descriptors
+// (SWIZZLE_128B, 8-row atoms of 1024 bytes) expect, so a block moves from HBM to
+// shared memory as one plain bulk copy and is consumed in place.
+// ---------------------------------------------------------------------------
+constexpr int kPage = 16;
+
+__host__ __device__ inline size_t block_bytes(int d) { return (size_t)kPage * d * 2; }
+__host__ __device__ inline size_t page_head_bytes(int d) { return 2 * block_bytes(d); }
+
+// byte offset of the 16-byte unit holding elements [8u', 8u'+8) of token t,
+// where e = element index in [0, d), inside a K or V block
+__host__ __device__ inline uint32_t unit_offset(int t, int e) {
+    int half = e >> 6;
+    int u = (e & 63) >> 3;
+    return (uint32_t)(half * 2048 + t * 128 + ((u ^ (t & 7)) << 4));
+}
+
+struct KvPool {
+    ps_shape shape;
+    int64_t num_pages;
+    char* base;
+    bool owned;
+    int32_t* meta_dev;   // q_start[n+1], prior[n] for ps_kv_write
+    int32_t meta_cap;    // ints
+    int32_t* flag_dev;   // bounds flag
+};
+
+const KvPool& pool_of(const ps_kv* kv);
+
+// ---------------------------------------------------------------------------
+// device work list
+// ---------------------------------------------------------------------------
+constexpr int kStatusOk = 0, kStatusBounds = 1, kStatusTimeout = 2;
+
+struct WsHeader {         // 64 bytes at the start of the workspace
+    int32_t status;       // sticky OR of kStatus* seen by any kernel of the run
+    int32_t decode_next;  // dynamic work counters
+    int32_t prefill_next;
+    int32_t pad[13];
+};
+
+// One contiguous page range of one (request, kv head) for the decode kernel.
+struct DecodePiece {
+    int32_t req;
+    int32_t kv_head;
+    int32_t page_begin;   // logical page indices within the request
+    int32_t page_end;
+    int32_t q_tok;        // packed q token index
+    int32_t part_slot;    // first partial slot (head 0 of the group), or -1: write final output
+    int32_t kv_len;       // keys visible to the row
+    int32_t pad;
+};
+
+// A decode work unit: pieces [piece_begin, piece_end) processed by one warp.
+struct DecodeUnit {
+    int32_t piece_begin;
+    int32_t piece_end;
+};
+
+// One q tile x key range of a prefill chunk for the prefill kernel.
+struct PrefillItem {
+    int32_t req;
+    int32_t kv_head;
+    int32_t key_begin;    // multiple of 128
+    int32_t key_end;      // exclusive; <= first_pos + n_tok
+    int32_t q_tok;        // packed index of the tile's first q token
+    int32_t n_tok;        // q tokens in the tile (<= 128 / G)
+    int32_t part_slot;    // partial slot of (segment, token 0, head 0), or -1: write final output
+    int32_t first_pos;    // absolute position of the tile's first q token (prior + index in chunk)
+};
+
+// Outputs that need the merge kernel: tokens [q_tok, q_tok + n_tok) x heads of
+// kv head g; partial (i, s, hh) is slot base + s * seg_stride + i * G + hh.
+struct MergeEntry {
+    int32_t q_tok;
+    int32_t n_tok;
+    int32_t kv_head;
+    int32_t base;
+    int32_t n_seg;
+    int32_t seg_stride;
+    int32_t pad[2];
+};
+
+struct DeviceWork {       // pointers into the workspace for one run
+    WsHeader* hdr;
+    const DecodePiece* pieces;
+    const DecodeUnit* units;
+    const PrefillItem* prefill;
+    const MergeEntry* merge;
+    float* part_lse;
+    float* part_o;
+    int32_t n_units, n_prefill, n_merge;
+};
+
+struct RunArgs {
+    ps_shape shape;
+    const char* pool;
+    int64_t num_pages;
+    const __nv_bfloat16* q;
+    const int32_t* block_table;
+    int32_t max_pages;
+    __nv_bfloat16* out;
+    float* lse;           // may be null
+    DeviceWork w;
+    cudaStream_t stream;
+    int num_sms;
+};
+
+ps_status launch_decode(const RunArgs& a);
+ps_status launch_prefill(const RunArgs& a);
+ps_status launch_merge(const RunArgs& a);
+int decode_warps_per_sm();
+
+// ---------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: returns false if the phase did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = 20000000u) {
+    for (uint32_t i = 0; i < limit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// global -> shared bulk copy; bytes multiple of 16, both addresses 16-byte aligned
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void fence_proxy_async_smem() {
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t x) {
+    uint32_t y;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+    return y;
+}
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace ps

@@ -1,0 +1,357 @@
+// Decode attention over the paged KV cache (rows with one new token).
+//
+// Decode attention streams every cached K and V of a request once and cannot
+// share those loads across requests (paper section 2.2), so it is bound by HBM
+// bandwidth.  Design for that bound:
+//   * each warp is an independent streaming engine with its own ring of
+//     shared-memory stages; one lane issues one bulk async copy per
+//     (page, kv head) block (K and V of 16 tokens, contiguous in the pool) and
+//     the warp waits on that stage's mbarrier -- no CTA-wide barrier anywhere;
+//   * the q heads that share a kv head ride in the N = 8 columns of
+//     mma.m16n8k16: S^T[16 tokens x heads] = K[16 x d] Q^T, then
+//     O^T[d x heads] += V^T[d x 16 tokens] P^T, so K and V are read from shared
+//     memory exactly once per group and no tensor-core row is padding at G = 8;
+//   * the softmax is over the token (row) axis of the accumulator fragment:
+//     two in-thread values plus three shuffles per head column;
+//   * P^T goes from accumulator layout to B-operand layout with movmatrix;
+//   * work arrives as equal-sized units of consecutive pages (possibly
+//     spanning several (request, kv head) pieces) fetched from one atomic
+//     counter; the producer side of the warp runs STAGES pages ahead of the
+//     consumer side, across piece and unit boundaries.
+#include "common.cuh"
+
+namespace ps {
+
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kRing = 8;  // unit ids in flight between the producer and consumer cursors of a warp
+
+template <int D>
+struct DecodeCfg {
+    static constexpr int kBlockBytes = kPage * D * 2;      // K (or V) of one page, one kv head
+    static constexpr int kStageBytes = 2 * kBlockBytes;    // K then V
+    static constexpr int kStages = (D == 128) ? 3 : 6;
+    static constexpr int kSmemBytes = kWarps * kStages * kStageBytes + kWarps * kStages * 8 + kWarps * kRing * 4 + 1024;
+};
+
+struct DecodeParams {
+    const char* pool;
+    int64_t num_pages;
+    const __nv_bfloat16* q;
+    const int32_t* block_table;
+    int32_t max_pages;
+    __nv_bfloat16* out;
+    float* lse;
+    WsHeader* hdr;
+    const DecodePiece* pieces;
+    const DecodeUnit* units;
+    int32_t n_units;
+    float* part_lse;
+    float* part_o;
+    int32_t Hq, Hkv, G;
+    float scale_log2;  // log2(e) / sqrt(d)
+};
+
+template <int D>
+__global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodeParams p) {
+    using Cfg = DecodeCfg<D>;
+    constexpr int STAGES = Cfg::kStages;
+    constexpr int KS = D / 16;  // k-steps of QK^T == m-tiles of PV
+
+    extern __shared__ char smem_raw[];
+    char* smem = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    char* my_stages = smem + (size_t)warp * STAGES * Cfg::kStageBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kWarps * STAGES * Cfg::kStageBytes) + warp * STAGES;
+    int32_t* ring = reinterpret_cast<int32_t*>(smem + (size_t)kWarps * STAGES * Cfg::kStageBytes + kWarps * STAGES * 8) +
+                    warp * kRing;
+    const uint32_t stage0 = smem_u32(my_stages);
+    const uint32_t bar0 = smem_u32(bars);
+
+    if (lane == 0) {
+        for (int s = 0; s < STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
+
+    // ---- producer cursor (warp-uniform) ----
+    bool P_done = false;
+    int P_piece = 0, P_piece_end = 0, P_page = 0, P_page_end = 0, P_g = 0, P_bt0 = 0, P_bt = 0;
+    const int32_t* P_row = p.block_table;
+    uint32_t n_prod = 0, pseq = 0;
+
+    auto produce = [&]() {
+        while (!P_done && P_page >= P_page_end) {
+            if (++P_piece >= P_piece_end) {
+                int u = 0;
+                if (lane == 0) u = atomicAdd(&p.hdr->decode_next, 1);
+                u = __shfl_sync(0xffffffffu, u, 0);
+                if (lane == 0) ring[pseq % kRing] = u;
+                ++pseq;
+                if (u >= p.n_units) { P_done = true; break; }
+                const DecodeUnit du = p.units[u];
+                P_piece = du.piece_begin;
+                P_piece_end = du.piece_end;
+            }
+            const int4 a = __ldg(reinterpret_cast<const int4*>(&p.pieces[P_piece]));
+            P_page = a.z;
+            P_page_end = a.w;
+            P_g = a.y;
+            P_row = p.block_table + (int64_t)a.x * p.max_pages;
+            P_bt0 = P_page;
+            P_bt = (P_bt0 + lane < P_page_end) ? __ldg(P_row + P_bt0 + lane) : 0;
+        }
+        if (P_done) return;
+        if (P_page >= P_bt0 + 32) {
+            P_bt0 += 32;
+            P_bt = (P_bt0 + lane < P_page_end) ? __ldg(P_row + P_bt0 + lane) : 0;
+        }
+        const int page = __shfl_sync(0xffffffffu, P_bt, P_page - P_bt0);
+        const uint32_t stage = n_prod % STAGES;
+        if (lane == 0) {
+            const uint32_t bar = bar0 + 8 * stage;
+            if ((uint32_t)page < (uint64_t)p.num_pages) {
+                mbar_expect_tx(bar, Cfg::kStageBytes);
+                bulk_g2s(stage0 + stage * Cfg::kStageBytes,
+                         p.pool + ((int64_t)page * p.Hkv + P_g) * (int64_t)Cfg::kStageBytes, Cfg::kStageBytes, bar);
+            } else {
+                atomicOr(&p.hdr->status, kStatusBounds);
+                mbar_arrive(bar);  // complete the phase without data; the run is flagged invalid
+            }
+        }
+        ++P_page;
+        ++n_prod;
+    };
+
+    for (int s = 0; s < STAGES; ++s) produce();
+
+    // ---- consumer cursor ----
+    int C_piece = 0, C_piece_end = 0, C_page = 0, C_page_end = 0;
+    int C_qtok = 0, C_slot = -1, C_kvlen = 0, C_g = 0;
+    bool have_piece = false, timed_out = false;
+    uint32_t n_cons = 0, cseq = 0;
+
+    uint32_t qb[KS][2];
+    float o[KS][4];
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+
+    const int col = 2 * (lane & 3);  // this thread's head columns: col, col + 1
+    const int row = lane >> 2;       // token rows row, row + 8 of S^T; d rows of O^T
+    const int mi = lane >> 3, l7 = lane & 7;
+    // ldmatrix row addresses (byte offsets inside a block, before the per-step unit term)
+    const uint32_t k_tok_off = (uint32_t)(((mi & 1) * 8 + l7) * 128);
+    const uint32_t v_tok_off = (uint32_t)(((mi >> 1) * 8 + l7) * 128);
+
+    auto finalize = [&]() {
+        // column sums over the 8 row-groups of the fragment
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 4);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 4);
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 8);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 8);
+        l0 += __shfl_xor_sync(0xffffffffu, l0, 16);
+        l1 += __shfl_xor_sync(0xffffffffu, l1, 16);
+        const float inv0 = 1.f / l0, inv1 = 1.f / l1;
+        const float lse0 = (m0 + log2f(l0)) * 0.6931471805599453f;
+        const float lse1 = (m1 + log2f(l1)) * 0.6931471805599453f;
+        const int h_base = C_g * p.G;
+        if (C_slot < 0) {
+            __nv_bfloat16* o0 = p.out + ((int64_t)C_qtok * p.Hq + h_base + col) * D;
+            __nv_bfloat16* o1 = o0 + D;
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) {
+                const int dd = mt * 16 + row;
+                if (col < p.G) {
+                    o0[dd] = __float2bfloat16_rn(o[mt][0] * inv0);
+                    o0[dd + 8] = __float2bfloat16_rn(o[mt][2] * inv0);
+                }
+                if (col + 1 < p.G) {
+                    o1[dd] = __float2bfloat16_rn(o[mt][1] * inv1);
+                    o1[dd + 8] = __float2bfloat16_rn(o[mt][3] * inv1);
+                }
+            }
+            if (p.lse && row == 0) {
+                if (col < p.G) p.lse[(int64_t)C_qtok * p.Hq + h_base + col] = lse0;
+                if (col + 1 < p.G) p.lse[(int64_t)C_qtok * p.Hq + h_base + col + 1] = lse1;
+            }
+        } else {
+            float* o0 = p.part_o + ((int64_t)C_slot + col) * D;
+            float* o1 = o0 + D;
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) {
+                const int dd = mt * 16 + row;
+                if (col < p.G) {
+                    o0[dd] = o[mt][0] * inv0;
+                    o0[dd + 8] = o[mt][2] * inv0;
+                }
+                if (col + 1 < p.G) {
+                    o1[dd] = o[mt][1] * inv1;
+                    o1[dd + 8] = o[mt][3] * inv1;
+                }
+            }
+            if (row == 0) {
+                if (col < p.G) p.part_lse[C_slot + col] = lse0;
+                if (col + 1 < p.G) p.part_lse[C_slot + col + 1] = lse1;
+            }
+        }
+    };
+
+    while (true) {
+        if (C_page >= C_page_end) {
+            if (have_piece) finalize();
+            have_piece = false;
+            if (++C_piece >= C_piece_end) {
+                __syncwarp();
+                const int u = ring[cseq % kRing];
+                ++cseq;
+                if (u >= p.n_units) break;
+                const DecodeUnit du = p.units[u];
+                C_piece = du.piece_begin;
+                C_piece_end = du.piece_end;
+            }
+            const int4 a = __ldg(reinterpret_cast<const int4*>(&p.pieces[C_piece]));
+            const int4 b = __ldg(reinterpret_cast<const int4*>(&p.pieces[C_piece]) + 1);
+            C_g = a.y;
+            C_page = a.z;
+            C_page_end = a.w;
+            C_qtok = b.x;
+            C_slot = b.y;
+            C_kvlen = b.z;
+            have_piece = true;
+            // Q^T as B fragments: thread holds head (lane / 4), d = 16 ks + 2 (lane % 4) + {0, 1} (+ 8)
+            const int hh = lane >> 2;
+            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q + ((int64_t)C_qtok * p.Hq + C_g * p.G + hh) * D);
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                qb[ks][0] = hh < p.G ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
+                qb[ks][1] = hh < p.G ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
+            }
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+            m0 = m1 = -INFINITY;
+            l0 = l1 = 0.f;
+        }
+
+        const uint32_t stage = n_cons % STAGES;
+        if (!mbar_wait(bar0 + 8 * stage, (n_cons / STAGES) & 1)) {
+            if (lane == 0) atomicOr(&p.hdr->status, kStatusTimeout);
+            timed_out = true;
+            break;
+        }
+        const uint32_t kbase = stage0 + stage * Cfg::kStageBytes;
+        const uint32_t vbase = kbase + Cfg::kBlockBytes;
+        const int nvalid = C_kvlen - C_page * kPage;  // >= 1
+
+        if (nvalid < kPage) {
+            // Slots past the sequence end hold whatever the pool holds (possibly NaN):
+            // zero those V rows so that 0 * V stays 0; their scores are masked below.
+            char* vb = my_stages + stage * Cfg::kStageBytes + Cfg::kBlockBytes;
+            const int units = (kPage - nvalid) * 8;  // 16-byte units per half
+            for (int h = 0; h < D / 64; ++h)
+                for (int u = lane; u < units; u += 32)
+                    *reinterpret_cast<uint4*>(vb + h * 2048 + nvalid * 128 + u * 16) = make_uint4(0, 0, 0, 0);
+            fence_proxy_async_smem();  // order these generic writes before the stage's next bulk copy
+            __syncwarp();
+        }
+
+        // S^T = K Q^T : 16 tokens x 8 head columns
+        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            const uint32_t unit = (uint32_t)(((ks * 2 + (mi >> 1)) & 7) ^ l7);
+            uint32_t a0, a1, a2, a3;
+            ldsm_x4(kbase + (ks >> 2) * 2048 + k_tok_off + (unit << 4), a0, a1, a2, a3);
+            if (ks & 1) mma_16816(sb, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+            else mma_16816(sa, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+        }
+        float x0 = (sa[0] + sb[0]) * p.scale_log2, x1 = (sa[1] + sb[1]) * p.scale_log2;
+        float x2 = (sa[2] + sb[2]) * p.scale_log2, x3 = (sa[3] + sb[3]) * p.scale_log2;
+        if (row >= nvalid) x0 = x1 = -INFINITY;
+        if (row + 8 >= nvalid) x2 = x3 = -INFINITY;
+
+        float mx0 = fmaxf(x0, x2), mx1 = fmaxf(x1, x3);
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 4));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 4));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 8));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 8));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 16));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 16));
+        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);  // finite: token 0 of the page is valid
+        const float al0 = fast_exp2(m0 - mn0), al1 = fast_exp2(m1 - mn1);
+        m0 = mn0;
+        m1 = mn1;
+        const float p0 = fast_exp2(x0 - mn0), p1 = fast_exp2(x1 - mn1);
+        const float p2 = fast_exp2(x2 - mn0), p3 = fast_exp2(x3 - mn1);
+        l0 = l0 * al0 + p0 + p2;
+        l1 = l1 * al1 + p1 + p3;
+        const uint32_t pb0 = movmatrix_t(pack_bf16(p0, p1));
+        const uint32_t pb1 = movmatrix_t(pack_bf16(p2, p3));
+
+        // O^T += V^T P^T : d x 8 head columns
+#pragma unroll
+        for (int mt = 0; mt < KS; ++mt) {
+            o[mt][0] *= al0;
+            o[mt][1] *= al1;
+            o[mt][2] *= al0;
+            o[mt][3] *= al1;
+            const uint32_t unit = (uint32_t)(((mt * 2 + (mi & 1)) & 7) ^ l7);
+            uint32_t a0, a1, a2, a3;
+            ldsm_x4_t(vbase + (mt >> 2) * 2048 + v_tok_off + (unit << 4), a0, a1, a2, a3);
+            mma_16816(o[mt], a0, a1, a2, a3, pb0, pb1);
+        }
+
+        __syncwarp();  // every lane has read this stage
+        ++C_page;
+        ++n_cons;
+        produce();     // refill the stage just released
+    }
+
+    if (timed_out) {
+        // let copies still in flight land before the CTA's shared memory is released
+        for (uint32_t n = n_cons + 1; n < n_prod; ++n) mbar_wait(bar0 + 8 * (n % STAGES), (n / STAGES) & 1, 2000000u);
+    }
+}
+
+}  // namespace
+
+int decode_warps_per_sm() { return kWarps; }
+
+template <int D>
+static ps_status launch_decode_d(const RunArgs& a) {
+    using Cfg = DecodeCfg<D>;
+    static bool configured = false;
+    if (!configured) {
+        PS_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+        configured = true;
+    }
+    DecodeParams p;
+    p.pool = a.pool;
+    p.num_pages = a.num_pages;
+    p.q = a.q;
+    p.block_table = a.block_table;
+    p.max_pages = a.max_pages;
+    p.out = a.out;
+    p.lse = a.lse;
+    p.hdr = a.w.hdr;
+    p.pieces = a.w.pieces;
+    p.units = a.w.units;
+    p.n_units = a.w.n_units;
+    p.part_lse = a.w.part_lse;
+    p.part_o = a.w.part_o;
+    p.Hq = a.shape.n_q_heads;
+    p.Hkv = a.shape.n_kv_heads;
+    p.G = p.Hq / p.Hkv;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+    int grid = (a.w.n_units + kWarps - 1) / kWarps;
+    if (grid > a.num_sms) grid = a.num_sms;
+    decode_kernel<D><<<grid, kWarps * 32, Cfg::kSmemBytes, a.stream>>>(p);
+    PS_CUDA_TRY(cudaGetLastError());
+    return PS_OK;
+}
+
+ps_status launch_decode(const RunArgs& a) {
+    if (a.w.n_units == 0) return PS_OK;
+    return a.shape.head_dim == 128 ? launch_decode_d<128>(a) : launch_decode_d<64>(a);
+}
+
+}  // namespace ps

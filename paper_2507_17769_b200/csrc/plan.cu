@@ -1,0 +1,407 @@
+// Host work partitioner and the per-iteration run entry point.
+//
+// The partition depends on the logical lengths only (never on page ids), so a
+// batch produces the same items, the same summation order and therefore the
+// same output bits under any assignment of physical pages.
+#include <algorithm>
+#include <chrono>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+namespace ps {
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+constexpr int kDecodeUnitsPerWarp = 2;  // dynamic-queue units per resident warp
+constexpr int kDecodeMinPages = 8;      // smallest decode unit (pages)
+constexpr int kPrefillKeyTile = 128;    // keys per tensor-core tile
+constexpr int kPrefillRows = 128;       // (token, head) rows per q tile
+
+}  // namespace ps
+
+using namespace ps;
+
+struct ps_plan {
+    ps_shape shape{};
+    int32_t n = 0, max_pages = 0, num_sms = 0, device_sms = 0;
+    std::vector<DecodePiece> pieces;
+    std::vector<DecodeUnit> units;
+    std::vector<PrefillItem> prefill;
+    std::vector<MergeEntry> merge;
+    std::vector<int32_t> prior;  // kept for item inspection
+    ps_plan_info info{};
+    // workspace layout
+    size_t off_pieces = 0, off_units = 0, off_prefill = 0, off_merge = 0, image_bytes = 0;
+    size_t off_part_lse = 0, off_part_o = 0, ws_bytes = 0;
+    // pinned staging image of [0, image_bytes)
+    char* pinned = nullptr;
+    bool pinned_is_cuda = false;
+    size_t pinned_cap = 0;
+    cudaEvent_t copied = nullptr;
+    bool copy_pending = false;
+    WsHeader* last_hdr = nullptr;
+};
+
+static int query_num_sms() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+    return sms;
+}
+
+static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len, const std::vector<int32_t>& q_start,
+                        const ps_plan_opts* opts, int64_t* n_slots) {
+    const int Hkv = pl->shape.n_kv_heads, G = pl->shape.n_q_heads / Hkv;
+    int64_t total_pages = 0;
+    for (int r = 0; r < pl->n; ++r)
+        if (q_len[r] == 1) total_pages += (int64_t)((prior[r] + 1 + kPage - 1) / kPage) * Hkv;
+    if (total_pages == 0) return;
+    int64_t per_unit;
+    if (opts && opts->decode_segment_tokens > 0) {
+        per_unit = std::max(1, opts->decode_segment_tokens / kPage);
+    } else {
+        const int64_t target = (int64_t)pl->num_sms * decode_warps_per_sm() * kDecodeUnitsPerWarp;
+        per_unit = std::max<int64_t>(kDecodeMinPages, (total_pages + target - 1) / target);
+    }
+    pl->info.decode_segment_tokens = (int32_t)(per_unit * kPage);
+
+    int64_t room = 0;  // pages the open unit can still take
+    for (int r = 0; r < pl->n; ++r) {
+        if (q_len[r] != 1) continue;
+        const int kv_len = prior[r] + 1;
+        const int pages = (kv_len + kPage - 1) / kPage;
+        for (int g = 0; g < Hkv; ++g) {
+            const size_t first_piece = pl->pieces.size();
+            int pg = 0;
+            while (pg < pages) {
+                if (room == 0) {
+                    pl->units.push_back(DecodeUnit{(int32_t)pl->pieces.size(), (int32_t)pl->pieces.size()});
+                    room = per_unit;
+                }
+                const int take = (int)std::min<int64_t>(room, pages - pg);
+                DecodePiece pc{};
+                pc.req = r;
+                pc.kv_head = g;
+                pc.page_begin = pg;
+                pc.page_end = pg + take;
+                pc.q_tok = q_start[r];
+                pc.part_slot = -1;
+                pc.kv_len = kv_len;
+                pl->pieces.push_back(pc);
+                pl->units.back().piece_end = (int32_t)pl->pieces.size();
+                pg += take;
+                room -= take;
+            }
+            const size_t cnt = pl->pieces.size() - first_piece;
+            if (cnt > 1) {
+                MergeEntry me{};
+                me.q_tok = q_start[r];
+                me.n_tok = 1;
+                me.kv_head = g;
+                me.base = (int32_t)*n_slots;
+                me.n_seg = (int32_t)cnt;
+                me.seg_stride = G;
+                pl->merge.push_back(me);
+                for (size_t s = 0; s < cnt; ++s) pl->pieces[first_piece + s].part_slot = (int32_t)(*n_slots + (int64_t)s * G);
+                *n_slots += (int64_t)cnt * G;
+            }
+        }
+    }
+}
+
+static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len, const std::vector<int32_t>& q_start,
+                         const ps_plan_opts* opts, int64_t* n_slots) {
+    const int Hkv = pl->shape.n_kv_heads, G = pl->shape.n_q_heads / Hkv;
+    const int tile_tok = kPrefillRows / G;
+    struct Tile { int r, g, tok0, n_tok, first_pos, key_tiles; };
+    std::vector<Tile> tiles;
+    int64_t total_key_tiles = 0;
+    for (int r = 0; r < pl->n; ++r) {
+        if (q_len[r] <= 1) continue;
+        for (int t0 = 0; t0 < q_len[r]; t0 += tile_tok) {
+            const int n_tok = std::min(tile_tok, q_len[r] - t0);
+            const int first_pos = prior[r] + t0;
+            const int kt = (first_pos + n_tok + kPrefillKeyTile - 1) / kPrefillKeyTile;
+            for (int g = 0; g < Hkv; ++g) {
+                tiles.push_back(Tile{r, g, t0, n_tok, first_pos, kt});
+                total_key_tiles += kt;
+            }
+        }
+    }
+    if (tiles.empty()) return;
+    int seg_tiles;  // key tiles per item
+    if (opts && opts->prefill_segment_tokens > 0) {
+        seg_tiles = std::max(1, opts->prefill_segment_tokens / kPrefillKeyTile);
+    } else if ((int64_t)tiles.size() >= 2LL * pl->num_sms) {
+        seg_tiles = 1 << 30;
+    } else {
+        const int64_t target = 2LL * pl->num_sms;
+        seg_tiles = (int)std::max<int64_t>(4, (total_key_tiles + target - 1) / target);
+    }
+    pl->info.prefill_segment_tokens = seg_tiles >= (1 << 22) ? 0 : seg_tiles * kPrefillKeyTile;
+
+    for (const Tile& t : tiles) {
+        const int n_seg = (t.key_tiles + seg_tiles - 1) / seg_tiles;
+        // spread the key tiles evenly over the segments
+        const int base_tiles = t.key_tiles / n_seg, extra = t.key_tiles % n_seg;
+        const int visible = t.first_pos + t.n_tok;
+        int32_t slot_base = -1;
+        if (n_seg > 1) {
+            slot_base = (int32_t)*n_slots;
+            MergeEntry me{};
+            me.q_tok = q_start[t.r] + t.tok0;
+            me.n_tok = t.n_tok;
+            me.kv_head = t.g;
+            me.base = slot_base;
+            me.n_seg = n_seg;
+            me.seg_stride = t.n_tok * G;
+            pl->merge.push_back(me);
+            *n_slots += (int64_t)n_seg * t.n_tok * G;
+        }
+        int kt0 = 0;
+        for (int s = 0; s < n_seg; ++s) {
+            const int nt = base_tiles + (s < extra ? 1 : 0);
+            PrefillItem it{};
+            it.req = t.r;
+            it.kv_head = t.g;
+            it.key_begin = kt0 * kPrefillKeyTile;
+            it.key_end = std::min(visible, (kt0 + nt) * kPrefillKeyTile);
+            it.q_tok = q_start[t.r] + t.tok0;
+            it.n_tok = t.n_tok;
+            it.part_slot = n_seg > 1 ? slot_base + s * t.n_tok * G : -1;
+            it.first_pos = t.first_pos;
+            pl->prefill.push_back(it);
+            kt0 += nt;
+        }
+    }
+    // longest first: the dynamic queue then finishes with the short items
+    std::stable_sort(pl->prefill.begin(), pl->prefill.end(), [](const PrefillItem& a, const PrefillItem& b) {
+        return (a.key_end - a.key_begin) > (b.key_end - b.key_begin);
+    });
+}
+
+extern "C" {
+
+ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const int32_t* q_len_host, int32_t n,
+                       int32_t max_pages_per_seq, const ps_plan_opts* opts, ps_plan** plan_inout,
+                       size_t* workspace_bytes_out) {
+    ps_status st = check_shape(shape);
+    if (st != PS_OK) return st;
+    if (!prior_host || !q_len_host || !plan_inout || !workspace_bytes_out) return fail(PS_ERR_INVALID, "null argument");
+    if (n < 1) return fail(PS_ERR_INVALID, "n=%d must be positive", n);
+    if (max_pages_per_seq < 1) return fail(PS_ERR_INVALID, "max_pages_per_seq=%d must be positive", max_pages_per_seq);
+    if (opts && (opts->decode_segment_tokens < 0 || opts->decode_segment_tokens % kPage != 0))
+        return fail(PS_ERR_INVALID, "decode_segment_tokens must be a non-negative multiple of %d", kPage);
+    if (opts && (opts->prefill_segment_tokens < 0 || opts->prefill_segment_tokens % kPrefillKeyTile != 0))
+        return fail(PS_ERR_INVALID, "prefill_segment_tokens must be a non-negative multiple of %d", kPrefillKeyTile);
+    std::vector<int32_t> q_start((size_t)n + 1);
+    int64_t T = 0;
+    for (int r = 0; r < n; ++r) {
+        if (q_len_host[r] < 1) return fail(PS_ERR_INVALID, "request %d: q_len=%d must be >= 1", r, q_len_host[r]);
+        if (prior_host[r] < 0) return fail(PS_ERR_INVALID, "request %d: prior=%d must be >= 0", r, prior_host[r]);
+        if ((int64_t)prior_host[r] + q_len_host[r] > (int64_t)max_pages_per_seq * kPage)
+            return fail(PS_ERR_INVALID, "request %d: kv_len=%lld exceeds max_pages_per_seq * page_size", r,
+                        (long long)prior_host[r] + q_len_host[r]);
+        q_start[r] = (int32_t)T;
+        T += q_len_host[r];
+        if (T > (1 << 24)) return fail(PS_ERR_INVALID, "more than 2^24 new tokens in one batch");
+    }
+    q_start[n] = (int32_t)T;
+
+    ps_plan* pl = *plan_inout;
+    const bool fresh = pl == nullptr;
+    if (fresh) {
+        pl = new (std::nothrow) ps_plan();
+        if (!pl) return fail(PS_ERR_OOM, "host allocation failed");
+    } else if (pl->copy_pending && pl->copied) {
+        cudaError_t e = cudaEventSynchronize(pl->copied);
+        if (e != cudaSuccess) return fail(PS_ERR_CUDA, "cudaEventSynchronize failed: %s", cudaGetErrorString(e));
+        pl->copy_pending = false;
+    }
+    pl->shape = *shape;
+    pl->n = n;
+    pl->max_pages = max_pages_per_seq;
+    if (opts && opts->num_sms > 0) {
+        pl->num_sms = opts->num_sms;
+    } else {
+        if (pl->device_sms <= 0) pl->device_sms = query_num_sms();
+        pl->num_sms = pl->device_sms;
+    }
+    if (pl->num_sms <= 0) {
+        if (fresh) delete pl;
+        return fail(PS_ERR_CUDA, "no CUDA device to plan for (pass opts->num_sms to plan without one)");
+    }
+    pl->pieces.clear();
+    pl->units.clear();
+    pl->prefill.clear();
+    pl->merge.clear();
+    pl->prior.assign(prior_host, prior_host + n);
+    pl->info = ps_plan_info{};
+    int64_t n_slots = 0;
+    plan_decode(pl, prior_host, q_len_host, q_start, opts, &n_slots);
+    plan_prefill(pl, prior_host, q_len_host, q_start, opts, &n_slots);
+    if (n_slots > 0x7fffffffLL) {
+        if (fresh) delete pl;
+        return fail(PS_ERR_UNSUPPORTED, "partial buffer would need %lld slots", (long long)n_slots);
+    }
+
+    const int d = shape->head_dim;
+    size_t off = 256;  // WsHeader
+    pl->off_pieces = off;   off = align_up(off + pl->pieces.size() * sizeof(DecodePiece), 256);
+    pl->off_units = off;    off = align_up(off + pl->units.size() * sizeof(DecodeUnit), 256);
+    pl->off_prefill = off;  off = align_up(off + pl->prefill.size() * sizeof(PrefillItem), 256);
+    pl->off_merge = off;    off = align_up(off + pl->merge.size() * sizeof(MergeEntry), 256);
+    pl->image_bytes = off;
+    pl->off_part_lse = off; off = align_up(off + (size_t)n_slots * sizeof(float), 256);
+    pl->off_part_o = off;   off = align_up(off + (size_t)n_slots * d * sizeof(float), 256);
+    pl->ws_bytes = off;
+
+    if (pl->pinned_cap < pl->image_bytes) {
+        if (pl->pinned) { if (pl->pinned_is_cuda) cudaFreeHost(pl->pinned); else free(pl->pinned); }
+        pl->pinned = nullptr;
+        const size_t cap = std::max(pl->image_bytes * 2, (size_t)1 << 16);
+        // Page-locked staging lets the work-list upload run asynchronously.  Without a CUDA
+        // device (planning ahead of time on another host) plain memory holds the image.
+        pl->pinned_is_cuda = cudaHostAlloc((void**)&pl->pinned, cap, cudaHostAllocDefault) == cudaSuccess;
+        if (!pl->pinned_is_cuda) {
+            (void)cudaGetLastError();
+            pl->pinned = (char*)malloc(cap);
+        }
+        if (!pl->pinned) {
+            pl->pinned_cap = 0;
+            if (fresh) delete pl;
+            return fail(PS_ERR_OOM, "cannot allocate %zu bytes of staging memory", cap);
+        }
+        pl->pinned_cap = cap;
+    }
+    if (!pl->copied && pl->pinned_is_cuda) {
+        if (cudaEventCreateWithFlags(&pl->copied, cudaEventDisableTiming) != cudaSuccess) {
+            (void)cudaGetLastError();
+            pl->copied = nullptr;
+        }
+    }
+    memset(pl->pinned, 0, 256);
+    if (!pl->pieces.empty()) memcpy(pl->pinned + pl->off_pieces, pl->pieces.data(), pl->pieces.size() * sizeof(DecodePiece));
+    if (!pl->units.empty()) memcpy(pl->pinned + pl->off_units, pl->units.data(), pl->units.size() * sizeof(DecodeUnit));
+    if (!pl->prefill.empty()) memcpy(pl->pinned + pl->off_prefill, pl->prefill.data(), pl->prefill.size() * sizeof(PrefillItem));
+    if (!pl->merge.empty()) memcpy(pl->pinned + pl->off_merge, pl->merge.data(), pl->merge.size() * sizeof(MergeEntry));
+
+    pl->info.n_decode_items = (int32_t)pl->pieces.size();
+    pl->info.n_prefill_items = (int32_t)pl->prefill.size();
+    int64_t merge_rows = 0;
+    for (const MergeEntry& me : pl->merge) merge_rows += (int64_t)me.n_tok * (shape->n_q_heads / shape->n_kv_heads);
+    pl->info.n_merge_rows = (int32_t)merge_rows;
+    pl->info.n_partial_slots = n_slots;
+    pl->info.total_q_tokens = T;
+    pl->info.n_launches = (pl->units.empty() ? 0 : 1) + (pl->prefill.empty() ? 0 : 1) + (pl->merge.empty() ? 0 : 1);
+    *plan_inout = pl;
+    *workspace_bytes_out = pl->ws_bytes;
+    return PS_OK;
+}
+
+ps_status ps_plan_free(ps_plan* pl) {
+    if (!pl) return PS_OK;
+    if (pl->copy_pending && pl->copied) cudaEventSynchronize(pl->copied);
+    if (pl->copied) cudaEventDestroy(pl->copied);
+    if (pl->pinned) { if (pl->pinned_is_cuda) cudaFreeHost(pl->pinned); else free(pl->pinned); }
+    delete pl;
+    return PS_OK;
+}
+
+ps_status ps_plan_get_info(const ps_plan* pl, ps_plan_info* info_out) {
+    if (!pl || !info_out) return fail(PS_ERR_INVALID, "null argument");
+    *info_out = pl->info;
+    return PS_OK;
+}
+
+ps_status ps_plan_get_items(const ps_plan* pl, int32_t* decode_items_out, int64_t decode_capacity,
+                            int32_t* prefill_items_out, int64_t prefill_capacity) {
+    if (!pl) return fail(PS_ERR_INVALID, "null argument");
+    if (decode_items_out) {
+        if (decode_capacity < (int64_t)pl->pieces.size()) return fail(PS_ERR_INVALID, "decode capacity too small");
+        for (size_t i = 0; i < pl->pieces.size(); ++i) {
+            const DecodePiece& pc = pl->pieces[i];
+            int32_t* o = decode_items_out + 8 * i;
+            o[0] = pc.req;
+            o[1] = pc.kv_head;
+            o[2] = pc.page_begin * kPage;
+            o[3] = std::min(pc.page_end * kPage, pc.kv_len);
+            o[4] = pc.q_tok;
+            o[5] = 1;
+            o[6] = pc.part_slot;
+            o[7] = pl->prior[pc.req];
+        }
+    }
+    if (prefill_items_out) {
+        if (prefill_capacity < (int64_t)pl->prefill.size()) return fail(PS_ERR_INVALID, "prefill capacity too small");
+        static_assert(sizeof(PrefillItem) == 32, "item record is 8 int32");
+        if (!pl->prefill.empty()) memcpy(prefill_items_out, pl->prefill.data(), pl->prefill.size() * sizeof(PrefillItem));
+    }
+    return PS_OK;
+}
+
+ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int32_t* block_table_dev, void* out_dev,
+                      float* lse_out_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    if (!pl || !kv || !q_dev || !block_table_dev || !out_dev || !workspace_dev) return fail(PS_ERR_INVALID, "null argument");
+    if (workspace_bytes < pl->ws_bytes)
+        return fail(PS_ERR_WORKSPACE, "workspace has %zu bytes, the plan needs %zu", workspace_bytes, pl->ws_bytes);
+    if ((uintptr_t)workspace_dev % 256 != 0) return fail(PS_ERR_INVALID, "workspace must be 256-byte aligned");
+    if (((uintptr_t)q_dev | (uintptr_t)out_dev) % 16 != 0) return fail(PS_ERR_INVALID, "q and out must be 16-byte aligned");
+    const KvPool& pool = pool_of(kv);
+    if (memcmp(&pool.shape, &pl->shape, sizeof(ps_shape)) != 0) return fail(PS_ERR_INVALID, "plan and pool shapes differ");
+    cudaStream_t s = (cudaStream_t)stream;
+    char* ws = (char*)workspace_dev;
+    PS_CUDA_TRY(cudaMemcpyAsync(ws, pl->pinned, pl->image_bytes, cudaMemcpyHostToDevice, s));
+    if (pl->copied) {
+        PS_CUDA_TRY(cudaEventRecord(pl->copied, s));
+        pl->copy_pending = true;
+    } else {
+        PS_CUDA_TRY(cudaStreamSynchronize(s));  // no event to guard the staging image: finish the copy now
+    }
+    pl->last_hdr = (WsHeader*)ws;
+
+    RunArgs a{};
+    a.shape = pl->shape;
+    a.pool = pool.base;
+    a.num_pages = pool.num_pages;
+    a.q = (const __nv_bfloat16*)q_dev;
+    a.block_table = block_table_dev;
+    a.max_pages = pl->max_pages;
+    a.out = (__nv_bfloat16*)out_dev;
+    a.lse = lse_out_dev;
+    a.stream = s;
+    a.num_sms = pl->num_sms;
+    a.w.hdr = (WsHeader*)ws;
+    a.w.pieces = (const DecodePiece*)(ws + pl->off_pieces);
+    a.w.units = (const DecodeUnit*)(ws + pl->off_units);
+    a.w.prefill = (const PrefillItem*)(ws + pl->off_prefill);
+    a.w.merge = (const MergeEntry*)(ws + pl->off_merge);
+    a.w.part_lse = (float*)(ws + pl->off_part_lse);
+    a.w.part_o = (float*)(ws + pl->off_part_o);
+    a.w.n_units = (int32_t)pl->units.size();
+    a.w.n_prefill = (int32_t)pl->prefill.size();
+    a.w.n_merge = (int32_t)pl->merge.size();
+
+    ps_status st = launch_prefill(a);
+    if (st != PS_OK) return st;
+    st = launch_decode(a);
+    if (st != PS_OK) return st;
+    return launch_merge(a);
+}
+
+ps_status ps_plan_status(ps_plan* pl, void* stream) {
+    if (!pl) return fail(PS_ERR_INVALID, "null argument");
+    PS_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    if (!pl->last_hdr) return PS_OK;
+    int32_t status = 0;
+    PS_CUDA_TRY(cudaMemcpy(&status, &pl->last_hdr->status, sizeof status, cudaMemcpyDeviceToHost));
+    if (status & kStatusTimeout) return fail(PS_ERR_TIMEOUT, "a bounded device-side wait expired; output is invalid");
+    if (status & kStatusBounds) return fail(PS_ERR_BOUNDS, "a block-table entry pointed outside the pool");
+    return PS_OK;
+}
+
+}  // extern "C"

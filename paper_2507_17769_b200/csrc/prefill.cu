@@ -1,0 +1,500 @@
+// Prefill-chunk attention on the 5th-generation tensor cores.
+//
+// A chunk's rows attend the prior context plus the chunk's own earlier tokens
+// (paper sections 2.4 and 4.7); this part is a dense contraction and compute
+// bound (section 3.4), so QK^T and PV run as tcgen05.mma with fp32
+// accumulators in tensor memory.
+//
+// One CTA works on one item = a q tile of 128 (token, head) rows that share a
+// kv head (the group's G heads of 128 / G consecutive tokens) x a key range.
+// Roles:
+//   warps 0-3  softmax: thread t owns row t (= TMEM lane t); reads S with
+//              tcgen05.ld, masks by the causal limit prior + i, keeps a
+//              running max with lazy rescaling of O, writes P (bf16) to shared
+//              memory in the operand layout, normalises and stores O at the end
+//   warp 4     producer: one 2 KB bulk async copy per (page, K|V, d half) into
+//              a 2-stage ring; the pool's page layout already is the
+//              128-byte-swizzled operand layout, so blocks are consumed in place
+//   warp 5     MMA issue: S[b] = Q K^T (8 x M128 N128 K16), O += P V
+//              (8 x M128 N=d K16), software-pipelined so QK^T of tile j+1
+//              overlaps the softmax of tile j; completion via tcgen05.commit
+// Every wait is bounded; on expiry the CTA sets the timeout status and drains.
+#include "common.cuh"
+
+namespace ps {
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kTileKeys = 128;
+constexpr int kRows = 128;
+constexpr float kRescaleThreshold = 8.f;  // log2 units
+
+// ---- tcgen05 wrappers -------------------------------------------------------
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle, 8-row atoms of 1024 bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version for this architecture
+    d |= (uint64_t)2 << 61;  // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(kRows >> 4) << 24);
+}
+
+template <int D>
+struct PrefillCfg {
+    static constexpr int kHalves = D / 64;
+    static constexpr int kHalfBytes = kTileKeys * 128;          // [128 rows][128 B]
+    static constexpr int kQBytes = kHalves * kHalfBytes;         // Q tile
+    static constexpr int kKBytes = kHalves * kHalfBytes;         // one K stage
+    static constexpr int kVBytes = kHalves * kHalfBytes;         // one V stage
+    static constexpr int kPBytes = 2 * kHalfBytes;               // P: two 64-key halves
+    static constexpr int kStages = 2;
+    static constexpr int kOffQ = 0;
+    static constexpr int kOffK = kOffQ + kQBytes;
+    static constexpr int kOffV = kOffK + kStages * kKBytes;
+    static constexpr int kOffP = kOffV + kStages * kVBytes;
+    static constexpr int kOffBar = kOffP + kPBytes;
+    static constexpr int kSmemBytes = kOffBar + 256 + 1024;      // + alignment slack
+    static constexpr int kTmemCols = 512;
+    static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256;
+};
+
+struct PrefillParams {
+    const char* pool;
+    int64_t num_pages;
+    const __nv_bfloat16* q;
+    const int32_t* block_table;
+    int32_t max_pages;
+    __nv_bfloat16* out;
+    float* lse;
+    WsHeader* hdr;
+    const PrefillItem* items;
+    int32_t n_items;
+    float* part_lse;
+    float* part_o;
+    int32_t Hq, Hkv, G;
+    float scale_log2;
+};
+
+struct Bars {  // byte offsets from the barrier block
+    static constexpr int k_full = 0, k_empty = 16, v_full = 32, v_empty = 48, s_full = 64, p_ready = 80, o_done = 88;
+    static constexpr int tmem_slot = 96, item_slot = 100, abort_slot = 104;
+};
+
+__device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < 40000000u; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+// warp-uniform result, so that the warp-collective instructions that follow stay converged
+__device__ __forceinline__ bool wait_all(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    return __all_sync(0xffffffffu, wait_or_abort(bar, parity, abort_flag));
+}
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParams p) {
+    using Cfg = PrefillCfg<D>;
+    extern __shared__ char smem_raw[];
+    char* smem = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t sbase = smem_u32(smem);
+    const uint32_t bars = sbase + Cfg::kOffBar;
+    volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + Cfg::kOffBar + Bars::tmem_slot);
+    volatile int* s_item = reinterpret_cast<volatile int*>(smem + Cfg::kOffBar + Bars::item_slot);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Cfg::kOffBar + Bars::abort_slot);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bars + Bars::k_full + 8 * s, 1);
+            mbar_init(bars + Bars::k_empty + 8 * s, 1);
+            mbar_init(bars + Bars::v_full + 8 * s, 1);
+            mbar_init(bars + Bars::v_empty + 8 * s, 1);
+            mbar_init(bars + Bars::s_full + 8 * s, 1);
+        }
+        mbar_init(bars + Bars::p_ready, kRows);
+        mbar_init(bars + Bars::o_done, 1);
+        mbar_fence_init();
+        *s_abort = 0;
+    }
+    if (warp == 0) {
+        tmem_alloc(bars + Bars::tmem_slot, Cfg::kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = (uint32_t)*s_tmem;
+
+    uint32_t tile_ctr = 0;  // key tiles processed by this CTA so far (every role counts the same)
+    constexpr uint32_t kIdescQK = instr_desc(kTileKeys, false);
+    constexpr uint32_t kIdescPV = instr_desc(D, true);
+
+    while (true) {
+        if (threadIdx.x == 0) *s_item = atomicAdd(&p.hdr->prefill_next, 1);
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        const int item_idx = *s_item;
+        if (item_idx >= p.n_items || *s_abort) break;
+        const PrefillItem it = p.items[item_idx];
+        const int n_tiles = (it.key_end - it.key_begin + kTileKeys - 1) / kTileKeys;
+
+        // ---- Q tile -> shared memory (row t = token t / G, head t % G) ----
+        if (warp < 4) {
+            const int t = threadIdx.x;
+            const int i = t / p.G, hh = t % p.G;
+            const bool valid = i < it.n_tok;
+            const uint4* src = reinterpret_cast<const uint4*>(
+                p.q + ((int64_t)(it.q_tok + (valid ? i : 0)) * p.Hq + it.kv_head * p.G + hh) * D);
+#pragma unroll
+            for (int U = 0; U < D / 8; ++U) {
+                const uint4 v = valid ? __ldg(src + U) : make_uint4(0, 0, 0, 0);
+                *reinterpret_cast<uint4*>(smem + Cfg::kOffQ + (U >> 3) * Cfg::kHalfBytes + t * 128 + (((U & 7) ^ (t & 7)) << 4)) = v;
+            }
+            fence_proxy_async_smem();
+        }
+        __syncthreads();
+
+        if (warp < 4) {
+            // =========================== softmax ===========================
+            const int t = threadIdx.x;
+            const int i = t / p.G;
+            const int limit = it.first_pos + i;  // last visible key of this row
+            const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+            float m = -INFINITY, l = 0.f;
+            bool ok = true;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const uint32_t tc = tile_ctr + j;
+                const uint32_t b = tc & 1;
+                ok = wait_all(bars + Bars::s_full + 8 * b, (tc >> 1) & 1, s_abort);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t s_addr = tmem + lane_addr + (b ? Cfg::kColS1 : Cfg::kColS0);
+                const int tile_base = it.key_begin + j * kTileKeys;
+                const bool need_mask = (tile_base + kTileKeys - 1 > it.first_pos) || (tile_base + kTileKeys > it.key_end);
+                const int vis = min(limit + 1, it.key_end) - tile_base;  // columns [0, vis) are visible to this row
+
+                // pass 1: row max of the raw scores
+                float mx = -INFINITY;
+#pragma unroll 1
+                for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(s_addr + c0, v);
+                    tmem_wait_ld();
+                    if (need_mask) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) mx = (c0 + c < vis) ? fmaxf(mx, __uint_as_float(v[c])) : mx;
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(v[c]));
+                    }
+                }
+                const float mx_s = mx * p.scale_log2;
+                float m_new = m;
+                if (mx_s > m + kRescaleThreshold || (m == -INFINITY && mx_s > -INFINITY)) m_new = mx_s;
+                const float alpha = (m_new == m) ? 1.f : fast_exp2(m - m_new);
+
+                if (j > 0) {
+                    // PV of the previous tile must be done before P is overwritten or O rescaled
+                    ok = wait_all(bars + Bars::o_done, (tc - 1) & 1, s_abort);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (__any_sync(0xffffffffu, m_new != m)) {
+#pragma unroll 1
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+                            uint32_t v[32];
+                            tmem_ld32(tmem + lane_addr + Cfg::kColO + c0, v);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) v[c] = __float_as_uint(__uint_as_float(v[c]) * alpha);
+                            tmem_st32(tmem + lane_addr + Cfg::kColO + c0, v);
+                        }
+                        tmem_wait_st();
+                    }
+                }
+                l *= alpha;
+                m = m_new;
+                const float m_sub = (m == -INFINITY) ? 0.f : m;
+
+                // pass 2: P = exp2(scale * s - m), bf16, into the A-operand layout
+#pragma unroll 1
+                for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(s_addr + c0, v);
+                    tmem_wait_ld();
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int c = 0; c < 32; c += 2) {
+                        float p0 = fast_exp2(fmaf(__uint_as_float(v[c]), p.scale_log2, -m_sub));
+                        float p1 = fast_exp2(fmaf(__uint_as_float(v[c + 1]), p.scale_log2, -m_sub));
+                        if (need_mask) {
+                            p0 = (c0 + c < vis) ? p0 : 0.f;
+                            p1 = (c0 + c + 1 < vis) ? p1 : 0.f;
+                        }
+                        l += p0 + p1;
+                        packed[c >> 1] = pack_bf16(p0, p1);
+                    }
+                    char* prow = smem + Cfg::kOffP + (c0 >> 6) * Cfg::kHalfBytes + t * 128;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        const int unit = ((c0 & 63) >> 3) + u;
+                        *reinterpret_cast<uint4*>(prow + ((unit ^ (t & 7)) << 4)) =
+                            make_uint4(packed[4 * u], packed[4 * u + 1], packed[4 * u + 2], packed[4 * u + 3]);
+                    }
+                }
+                // keys at or past key_end: their V rows may be stale or poisoned; zero them so 0 * V = 0
+                const int n_keys = it.key_end - tile_base;
+                if (n_keys < kTileKeys) {
+                    ok = wait_all(bars + Bars::v_full + 8 * b, (tc >> 1) & 1, s_abort);
+                    if (!ok) break;
+                    if (t >= n_keys) {
+                        char* vrow = smem + Cfg::kOffV + b * Cfg::kVBytes + t * 128;
+#pragma unroll
+                        for (int h = 0; h < Cfg::kHalves; ++h)
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                *reinterpret_cast<uint4*>(vrow + h * Cfg::kHalfBytes + u * 16) = make_uint4(0, 0, 0, 0);
+                    }
+                }
+                fence_proxy_async_smem();
+                tc_fence_before();
+                mbar_arrive(bars + Bars::p_ready);
+            }
+            // ---- epilogue: O / l ----
+            if (ok) ok = wait_all(bars + Bars::o_done, (tile_ctr + n_tiles - 1) & 1, s_abort);
+            if (ok) {
+                tc_fence_after();
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+                const float lse_v = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                const bool valid = i < it.n_tok;
+                const int hh = t % p.G;
+                const int64_t orow = (int64_t)(it.q_tok + i) * p.Hq + it.kv_head * p.G + hh;
+#pragma unroll 1
+                for (int c0 = 0; c0 < D; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem + lane_addr + Cfg::kColO + c0, v);
+                    tmem_wait_ld();
+                    if (!valid) continue;
+                    if (it.part_slot < 0) {
+                        uint4* dst = reinterpret_cast<uint4*>(p.out + orow * D + c0);
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            uint4 w;
+                            w.x = pack_bf16(__uint_as_float(v[8 * u + 0]) * inv, __uint_as_float(v[8 * u + 1]) * inv);
+                            w.y = pack_bf16(__uint_as_float(v[8 * u + 2]) * inv, __uint_as_float(v[8 * u + 3]) * inv);
+                            w.z = pack_bf16(__uint_as_float(v[8 * u + 4]) * inv, __uint_as_float(v[8 * u + 5]) * inv);
+                            w.w = pack_bf16(__uint_as_float(v[8 * u + 6]) * inv, __uint_as_float(v[8 * u + 7]) * inv);
+                            dst[u] = w;
+                        }
+                    } else {
+                        float4* dst = reinterpret_cast<float4*>(p.part_o + ((int64_t)it.part_slot + t) * D + c0);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            dst[u] = make_float4(__uint_as_float(v[4 * u]) * inv, __uint_as_float(v[4 * u + 1]) * inv,
+                                                 __uint_as_float(v[4 * u + 2]) * inv, __uint_as_float(v[4 * u + 3]) * inv);
+                    }
+                }
+                if (valid) {
+                    if (it.part_slot < 0) {
+                        if (p.lse) p.lse[orow] = lse_v;
+                    } else {
+                        p.part_lse[it.part_slot + t] = lse_v;
+                    }
+                }
+            }
+        } else if (warp == 4) {
+            // =========================== producer ===========================
+            const int pg = lane >> 2, which = lane & 3;  // page in tile; 0/1 = K half 0/1, 2/3 = V half 0/1
+            const int32_t* bt = p.block_table + (int64_t)it.req * p.max_pages + it.key_begin / kPage;
+            constexpr uint32_t kPieceBytes = kPage * 128;  // 16 tokens x 64 elements
+            bool ok = true;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const uint32_t tc = tile_ctr + j;
+                const uint32_t s = tc & 1, par = (tc >> 1) & 1;
+                const int n_keys = min(kTileKeys, it.key_end - (it.key_begin + j * kTileKeys));
+                const int n_pages = (n_keys + kPage - 1) / kPage;
+                int page = (lane < n_pages) ? __ldg(bt + j * 8 + lane) : 0;
+                const bool in_range = (uint32_t)page < (uint64_t)p.num_pages;
+                const uint32_t good = __ballot_sync(0xffffffffu, lane < n_pages && in_range);
+                if (__popc(good) != n_pages && lane == 0) atomicOr(&p.hdr->status, kStatusBounds);
+                const int my_page = __shfl_sync(0xffffffffu, page, pg);
+                const bool mine = (good >> pg) & 1u;
+                const uint32_t tile_bytes = (uint32_t)__popc(good) * Cfg::kHalves * kPieceBytes;
+                const char* src = p.pool + ((int64_t)my_page * p.Hkv + it.kv_head) * (int64_t)(2 * Cfg::kHalves * kPieceBytes);
+
+                ok = wait_all(bars + Bars::k_empty + 8 * s, par ^ 1, s_abort);
+                if (!ok) break;
+                if (lane == 0) mbar_expect_tx(bars + Bars::k_full + 8 * s, tile_bytes);
+                __syncwarp();
+                if (mine && which < Cfg::kHalves)
+                    bulk_g2s(sbase + Cfg::kOffK + s * Cfg::kKBytes + which * Cfg::kHalfBytes + pg * kPieceBytes,
+                             src + which * kPieceBytes, kPieceBytes, bars + Bars::k_full + 8 * s);
+
+                ok = wait_all(bars + Bars::v_empty + 8 * s, par ^ 1, s_abort);
+                if (!ok) break;
+                if (lane == 0) mbar_expect_tx(bars + Bars::v_full + 8 * s, tile_bytes);
+                __syncwarp();
+                if (mine && which >= 2 && which - 2 < Cfg::kHalves)
+                    bulk_g2s(sbase + Cfg::kOffV + s * Cfg::kVBytes + (which - 2) * Cfg::kHalfBytes + pg * kPieceBytes,
+                             src + (Cfg::kHalves + which - 2) * kPieceBytes, kPieceBytes, bars + Bars::v_full + 8 * s);
+            }
+        } else {
+            // =========================== MMA issue ===========================
+            bool ok = true;
+            auto issue_qk = [&](int j) {
+                const uint32_t tc = tile_ctr + j;
+                const uint32_t s = tc & 1;
+                ok = wait_all(bars + Bars::k_full + 8 * s, (tc >> 1) & 1, s_abort);
+                if (!ok) return;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t d_addr = tmem + (s ? Cfg::kColS1 : Cfg::kColS0);
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = (kk >> 2) * Cfg::kHalfBytes + (kk & 3) * 32;
+                        tc_mma_ss(d_addr, smem_desc(sbase + Cfg::kOffQ + off, 16, 1024),
+                                  smem_desc(sbase + Cfg::kOffK + s * Cfg::kKBytes + off, 16, 1024), kIdescQK, kk > 0);
+                    }
+                    tc_commit(bars + Bars::s_full + 8 * s);
+                    tc_commit(bars + Bars::k_empty + 8 * s);
+                }
+                __syncwarp();
+            };
+            issue_qk(0);
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                if (j + 1 < n_tiles) issue_qk(j + 1);
+                if (!ok) break;
+                const uint32_t tc = tile_ctr + j;
+                const uint32_t s = tc & 1;
+                ok = wait_all(bars + Bars::p_ready, tc & 1, s_abort);
+                if (!ok) break;
+                ok = wait_all(bars + Bars::v_full + 8 * s, (tc >> 1) & 1, s_abort);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+#pragma unroll
+                    for (int kk = 0; kk < kTileKeys / 16; ++kk) {
+                        const uint64_t a = smem_desc(sbase + Cfg::kOffP + (kk >> 2) * Cfg::kHalfBytes + (kk & 3) * 32, 16, 1024);
+                        const uint64_t bdesc = smem_desc(sbase + Cfg::kOffV + s * Cfg::kVBytes + kk * 2048, Cfg::kHalfBytes, 1024);
+                        tc_mma_ss(tmem + Cfg::kColO, a, bdesc, kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit(bars + Bars::o_done);
+                    tc_commit(bars + Bars::v_empty + 8 * s);
+                }
+                __syncwarp();
+            }
+        }
+        tile_ctr += n_tiles;
+    }
+
+    // after an abort: flag the run and give copies in flight a bounded time to land
+    if (*s_abort) {
+        if (threadIdx.x == 0) atomicOr(&p.hdr->status, kStatusTimeout);
+        for (int s = 0; s < 2; ++s) {
+            mbar_wait(bars + Bars::k_full + 8 * s, 0, 200000u);
+            mbar_wait(bars + Bars::v_full + 8 * s, 0, 200000u);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
+}
+
+}  // namespace
+
+template <int D>
+static ps_status launch_prefill_d(const RunArgs& a) {
+    using Cfg = PrefillCfg<D>;
+    static bool configured = false;
+    if (!configured) {
+        PS_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+        configured = true;
+    }
+    PrefillParams p;
+    p.pool = a.pool;
+    p.num_pages = a.num_pages;
+    p.q = a.q;
+    p.block_table = a.block_table;
+    p.max_pages = a.max_pages;
+    p.out = a.out;
+    p.lse = a.lse;
+    p.hdr = a.w.hdr;
+    p.items = a.w.prefill;
+    p.n_items = a.w.n_prefill;
+    p.part_lse = a.w.part_lse;
+    p.part_o = a.w.part_o;
+    p.Hq = a.shape.n_q_heads;
+    p.Hkv = a.shape.n_kv_heads;
+    p.G = p.Hq / p.Hkv;
+    p.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+    const int grid = a.w.n_prefill < a.num_sms ? a.w.n_prefill : a.num_sms;
+    prefill_kernel<D><<<grid, kThreads, Cfg::kSmemBytes, a.stream>>>(p);
+    PS_CUDA_TRY(cudaGetLastError());
+    return PS_OK;
+}
+
+ps_status launch_prefill(const RunArgs& a) {
+    if (a.w.n_prefill == 0) return PS_OK;
+    return a.shape.head_dim == 128 ? launch_prefill_d<128>(a) : launch_prefill_d<64>(a);
+}
+
+}  // namespace ps

@@ -1,0 +1,170 @@
+"""CPU-side checks of the C-ABI library: it loads, exports what the header
+declares, validates arguments, and the host partitioner covers every
+(query row, visible key) exactly once.  No kernel is launched here."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2507_17769_b200 as ps
+from paper_2507_17769_b200 import binding as B
+from workloads import gen
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def opts(num_sms=148, dec=0, pre=0):
+    return ps.ps_plan_opts(dec, pre, num_sms)
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "polyserve_attn.h")).read()
+    declared = set(re.findall(r"\b(ps_[a-z_]+)\s*\(", header))
+    assert declared == set(B.EXPORTS)
+    lib = B.load()
+    for name in declared:
+        assert getattr(lib, name) is not None
+    assert "sm_100a" in ps.ps_version()
+
+
+def test_kv_bytes_and_shape_validation():
+    s = ps.make_shape(32, 8, 128)
+    assert ps.ps_kv_bytes(s, 10) == 10 * 8 * 2 * 16 * 128 * 2
+    assert ps.ps_kv_bytes(ps.make_shape(4, 2, 64), 3) == 3 * 2 * 2 * 16 * 64 * 2
+    for bad, code in [((32, 8, 96, 16), B.PS_ERR_UNSUPPORTED), ((32, 8, 128, 32), B.PS_ERR_UNSUPPORTED),
+                      ((32, 5, 128, 16), B.PS_ERR_INVALID), ((48, 1, 128, 16), B.PS_ERR_UNSUPPORTED)]:
+        with pytest.raises(ps.PsError) as e:
+            ps.ps_kv_bytes(ps.make_shape(*bad), 4)
+        assert e.value.status == code
+    with pytest.raises(ps.PsError):
+        ps.ps_kv_bytes(s, 0)
+
+
+def test_plan_rejects_bad_lengths():
+    s = ps.make_shape(32, 8, 128)
+    for prior, q_len, max_pages in [([5], [0], 4), ([-1], [1], 4), ([100], [1], 4), ([0], [65], 4)]:
+        with pytest.raises(ps.PsError) as e:
+            ps.ps_attn_plan(s, prior, q_len, max_pages, opts())
+        assert e.value.status == B.PS_ERR_INVALID
+    with pytest.raises(ps.PsError):
+        ps.ps_attn_plan(s, [5], [1], 4, opts(dec=24))  # not a multiple of the page size
+
+
+def coverage_check(batch, plan):
+    """Every (request, kv head, q token, key <= causal limit) is covered by exactly one item."""
+    s = batch.shape
+    G = s.group
+    dec, pre = ps.ps_plan_get_items(plan)
+    q_start = batch.q_start
+    # decode: per (req, kv head) the pieces tile [0, kv_len) in order
+    seen = {}
+    for it in dec:
+        r, g, k0, k1, qt, nt, slot, fp = it.tolist()
+        assert batch.q_len[r] == 1 and nt == 1 and qt == q_start[r] and fp == batch.prior[r]
+        assert k0 % 16 == 0 and k0 < k1 <= batch.kv_len[r]
+        seen.setdefault((r, g), []).append((k0, k1, slot))
+    for r in range(batch.n):
+        if batch.q_len[r] != 1:
+            continue
+        for g in range(s.n_kv_heads):
+            segs = sorted(seen[(r, g)])
+            assert segs[0][0] == 0 and segs[-1][1] == batch.kv_len[r]
+            for a, b in zip(segs[:-1], segs[1:]):
+                assert a[1] == b[0]
+            slots = [x[2] for x in segs]
+            if len(segs) == 1:
+                assert slots == [-1]
+            else:
+                assert all(x >= 0 for x in slots) and [x - slots[0] for x in slots] == [i * G for i in range(len(slots))]
+    # prefill: per (req, kv head, tile) the segments tile [0, first_pos + n_tok)
+    tiles = {}
+    for it in pre:
+        r, g, k0, k1, qt, nt, slot, fp = it.tolist()
+        assert batch.q_len[r] > 1 and k0 % 128 == 0 and k0 < k1
+        tok0 = qt - q_start[r]
+        assert fp == batch.prior[r] + tok0 and 1 <= nt <= 128 // G and tok0 % (128 // G) == 0
+        assert k1 <= fp + nt
+        tiles.setdefault((r, g, tok0, nt), []).append((k0, k1, slot))
+    for r in range(batch.n):
+        c = int(batch.q_len[r])
+        if c <= 1:
+            continue
+        tt = 128 // G
+        for g in range(s.n_kv_heads):
+            covered = 0
+            for tok0 in range(0, c, tt):
+                nt = min(tt, c - tok0)
+                segs = sorted(tiles[(r, g, tok0, nt)])
+                assert segs[0][0] == 0 and segs[-1][1] == batch.prior[r] + tok0 + nt
+                for a, b in zip(segs[:-1], segs[1:]):
+                    assert a[1] == b[0]
+                if len(segs) == 1:
+                    assert segs[0][2] == -1
+                else:
+                    base = segs[0][2]
+                    assert [x[2] - base for x in segs] == [i * nt * G for i in range(len(segs))]
+                covered += nt
+            assert covered == c
+    # partial slots of different groups never overlap
+    info = ps.ps_plan_get_info(plan)
+    used = np.zeros(info.n_partial_slots, dtype=np.int32)
+    for (r, g), segs in seen.items():
+        for k0, k1, slot in segs:
+            if slot >= 0:
+                used[slot : slot + G] += 1
+    for (r, g, tok0, nt), segs in tiles.items():
+        for k0, k1, slot in segs:
+            if slot >= 0:
+                used[slot : slot + nt * G] += 1
+    assert np.all(used == 1)
+    return info
+
+
+@pytest.mark.parametrize("make,kw", [
+    (gen.config0, {}), (gen.config0, {"dec": 16, "pre": 128}), (gen.config1, {}), (gen.config2, {}),
+    (lambda: gen.config3_cell(64, 8, 8192, 3001), {}), (lambda: gen.config3_cell(2048, 256, 512, 3002), {}),
+    (gen.config4, {}),
+])
+def test_partition_covers_every_row_and_key_once(make, kw):
+    batch = make()
+    sh = ps.make_shape(batch.shape.n_q_heads, batch.shape.n_kv_heads, batch.shape.head_dim)
+    plan, ws = ps.ps_attn_plan(sh, batch.prior, batch.q_len, batch.max_pages, opts(**kw))
+    try:
+        info = coverage_check(batch, plan)
+        assert info.total_q_tokens == batch.total_q
+        assert ws >= 256 + info.n_partial_slots * (batch.shape.head_dim + 1) * 4
+    finally:
+        ps.ps_plan_free(plan)
+
+
+def test_partition_ignores_page_ids_and_replans_in_place():
+    b = gen.config2()
+    sh = ps.make_shape(32, 8, 128)
+    plan, ws1 = ps.ps_attn_plan(sh, b.prior, b.q_len, b.max_pages, opts())
+    d1, p1 = ps.ps_plan_get_items(plan)
+    plan2, ws2 = ps.ps_attn_plan(sh, b.prior, b.q_len, b.max_pages + 7, opts())
+    d2, p2 = ps.ps_plan_get_items(plan2)
+    assert np.array_equal(d1, d2) and np.array_equal(p1, p2) and ws1 == ws2
+    # rebuild the first handle for another batch, then back: same items again
+    c = gen.config1()
+    same, _ = ps.ps_attn_plan(sh, c.prior, c.q_len, c.max_pages, opts(), plan)
+    assert same == plan and ps.ps_plan_get_info(plan).n_prefill_items == 0
+    ps.ps_attn_plan(sh, b.prior, b.q_len, b.max_pages, opts(), plan)
+    d3, p3 = ps.ps_plan_get_items(plan)
+    assert np.array_equal(d1, d3) and np.array_equal(p1, p3)
+    ps.ps_plan_free(plan)
+    ps.ps_plan_free(plan2)
+
+
+def test_decode_units_are_balanced():
+    b = gen.config1()
+    sh = ps.make_shape(32, 8, 128)
+    plan, _ = ps.ps_attn_plan(sh, b.prior, b.q_len, b.max_pages, opts())
+    info = ps.ps_plan_get_info(plan)
+    total_pages = int(((b.kv_len + 15) // 16).sum()) * 8
+    per_unit = info.decode_segment_tokens // 16
+    assert per_unit == max(8, -(-total_pages // (148 * 8 * 2)))
+    # partial rows stay a small fraction of the KV stream
+    assert info.n_partial_slots * 128 * 4 < 0.1 * b.decode_bytes()
+    ps.ps_plan_free(plan)
