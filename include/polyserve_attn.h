@@ -196,6 +196,21 @@ ps_status ps_attn_run(ps_plan *plan, const ps_kv *kv, const void *q_dev, const i
  * skipped) or PS_ERR_TIMEOUT (a bounded wait expired; output is invalid). */
 ps_status ps_plan_status(ps_plan *plan, void *stream);
 
+/*
+ * Per-kernel timing of the next runs of this plan (the profile of section 4.5
+ * split into its prefill-attention and decode-attention terms, section 3.4).
+ * ps_plan_set_timing(plan, max_runs) makes each of the next max_runs calls of
+ * ps_attn_run record CUDA events on its stream around the prefill, decode and
+ * merge launches (max_runs = 0 switches recording off); calling it again
+ * restarts the count.  ps_plan_get_timing synchronises `stream` and returns
+ * the mean duration in milliseconds of each kernel over the runs recorded so
+ * far, and how many there were.  A kernel the plan does not launch reports the
+ * (near-zero) gap between its two events.
+ */
+ps_status ps_plan_set_timing(ps_plan *plan, int32_t max_runs);
+ps_status ps_plan_get_timing(ps_plan *plan, void *stream, float *prefill_ms_out, float *decode_ms_out,
+                             float *merge_ms_out, int32_t *n_runs_out);
+
 /* ------------------------------------------------------------------------ */
 /* Latency-table sweep (section 4.5: a profiled map from batch size and KV    */
 /* cache size to execution time, which the scheduler consults).               */

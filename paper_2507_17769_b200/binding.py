@@ -62,7 +62,8 @@ class ps_grid_row(ctypes.Structure):
 
 
 EXPORTS = ["ps_kv_bytes", "ps_kv_alloc", "ps_kv_free", "ps_kv_write", "ps_kv_gather", "ps_kv_status", "ps_attn_plan",
-           "ps_plan_free", "ps_plan_get_info", "ps_plan_get_items", "ps_attn_run", "ps_plan_status", "ps_profile_grid",
+           "ps_plan_free", "ps_plan_get_info", "ps_plan_get_items", "ps_attn_run", "ps_plan_status",
+           "ps_plan_set_timing", "ps_plan_get_timing", "ps_profile_grid",
            "ps_last_error", "ps_version"]
 
 _lib = None
@@ -93,6 +94,9 @@ def load() -> ctypes.CDLL:
     lib.ps_plan_get_items.argtypes = [_vp, _i32p, _i64, _i32p, _i64]
     lib.ps_attn_run.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
     lib.ps_plan_status.argtypes = [_vp, _vp]
+    lib.ps_plan_set_timing.argtypes = [_vp, _i32]
+    fp = ctypes.POINTER(ctypes.c_float)
+    lib.ps_plan_get_timing.argtypes = [_vp, _vp, fp, fp, fp, ctypes.POINTER(_i32)]
     lib.ps_profile_grid.argtypes = [sp, ctypes.POINTER(ps_grid_spec), ctypes.POINTER(ps_grid_row), _i64,
                                     ctypes.POINTER(_i64), ctypes.c_char_p, _vp]
     for name in EXPORTS:
@@ -204,6 +208,17 @@ def ps_attn_run(plan, kv, q_dev, block_table_dev, out_dev, lse_out_dev, workspac
 
 def ps_plan_status(plan, stream=None):
     _check(load().ps_plan_status(plan, _ptr(stream)))
+
+
+def ps_plan_set_timing(plan, max_runs: int):
+    _check(load().ps_plan_set_timing(plan, max_runs))
+
+
+def ps_plan_get_timing(plan, stream=None):
+    """Returns (prefill_ms, decode_ms, merge_ms, n_runs): mean per-kernel time of the recorded runs."""
+    a, b, c, n = ctypes.c_float(0), ctypes.c_float(0), ctypes.c_float(0), _i32(0)
+    _check(load().ps_plan_get_timing(plan, _ptr(stream), ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(n)))
+    return a.value, b.value, c.value, n.value
 
 
 def ps_profile_grid(shape: ps_shape, chunk_sizes, decode_counts, mean_ctxs, seeds_per_cell, warmup, iters, seed_base,

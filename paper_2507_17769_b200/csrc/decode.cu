@@ -282,10 +282,13 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
         m1 = mn1;
         const float p0 = fast_exp2(x0 - mn0), p1 = fast_exp2(x1 - mn1);
         const float p2 = fast_exp2(x2 - mn0), p3 = fast_exp2(x3 - mn1);
-        l0 = l0 * al0 + p0 + p2;
-        l1 = l1 * al1 + p1 + p3;
-        const uint32_t pb0 = movmatrix_t(pack_bf16(p0, p1));
-        const uint32_t pb1 = movmatrix_t(pack_bf16(p2, p3));
+        // the row sum uses the bf16-rounded weights that PV multiplies, so that the
+        // normalised output is an exact convex mix of V rows
+        const uint32_t pk0 = pack_bf16(p0, p1), pk1 = pack_bf16(p2, p3);
+        l0 = l0 * al0 + bf16_lo(pk0) + bf16_lo(pk1);
+        l1 = l1 * al1 + bf16_hi(pk0) + bf16_hi(pk1);
+        const uint32_t pb0 = movmatrix_t(pk0);
+        const uint32_t pb1 = movmatrix_t(pk1);
 
         // O^T += V^T P^T : d x 8 head columns
 #pragma unroll

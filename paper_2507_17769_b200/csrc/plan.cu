@@ -44,6 +44,10 @@ struct ps_plan {
     cudaEvent_t copied = nullptr;
     bool copy_pending = false;
     WsHeader* last_hdr = nullptr;
+    // optional per-kernel timing: 4 events per recorded run (before prefill, after prefill, after decode, after merge)
+    bool timing = false;
+    std::vector<cudaEvent_t> tev;
+    int timed_runs = 0;
 };
 
 static int query_num_sms() {
@@ -307,6 +311,7 @@ ps_status ps_plan_free(ps_plan* pl) {
     if (!pl) return PS_OK;
     if (pl->copy_pending && pl->copied) cudaEventSynchronize(pl->copied);
     if (pl->copied) cudaEventDestroy(pl->copied);
+    for (cudaEvent_t e : pl->tev) cudaEventDestroy(e);
     if (pl->pinned) { if (pl->pinned_is_cuda) cudaFreeHost(pl->pinned); else free(pl->pinned); }
     delete pl;
     return PS_OK;
@@ -386,11 +391,53 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     a.w.n_prefill = (int32_t)pl->prefill.size();
     a.w.n_merge = (int32_t)pl->merge.size();
 
+    const bool rec = pl->timing && (size_t)(pl->timed_runs + 1) * 4 <= pl->tev.size();
+    cudaEvent_t* ev = rec ? &pl->tev[(size_t)pl->timed_runs * 4] : nullptr;
+    if (rec) cudaEventRecord(ev[0], s);
     ps_status st = launch_prefill(a);
     if (st != PS_OK) return st;
+    if (rec) cudaEventRecord(ev[1], s);
     st = launch_decode(a);
     if (st != PS_OK) return st;
-    return launch_merge(a);
+    if (rec) cudaEventRecord(ev[2], s);
+    st = launch_merge(a);
+    if (rec) {
+        cudaEventRecord(ev[3], s);
+        ++pl->timed_runs;
+    }
+    return st;
+}
+
+ps_status ps_plan_set_timing(ps_plan* pl, int32_t max_runs) {
+    if (!pl) return fail(PS_ERR_INVALID, "null argument");
+    if (max_runs < 0 || max_runs > 4096) return fail(PS_ERR_INVALID, "max_runs=%d outside [0, 4096]", max_runs);
+    pl->timed_runs = 0;
+    pl->timing = max_runs > 0;
+    while (pl->tev.size() < (size_t)max_runs * 4) {
+        cudaEvent_t e;
+        PS_CUDA_TRY(cudaEventCreate(&e));
+        pl->tev.push_back(e);
+    }
+    return PS_OK;
+}
+
+ps_status ps_plan_get_timing(ps_plan* pl, void* stream, float* prefill_ms_out, float* decode_ms_out, float* merge_ms_out,
+                             int32_t* n_runs_out) {
+    if (!pl || !prefill_ms_out || !decode_ms_out || !merge_ms_out || !n_runs_out) return fail(PS_ERR_INVALID, "null argument");
+    PS_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    double acc[3] = {0, 0, 0};
+    for (int r = 0; r < pl->timed_runs; ++r)
+        for (int k = 0; k < 3; ++k) {
+            float ms = 0.f;
+            PS_CUDA_TRY(cudaEventElapsedTime(&ms, pl->tev[(size_t)r * 4 + k], pl->tev[(size_t)r * 4 + k + 1]));
+            acc[k] += ms;
+        }
+    const double n = pl->timed_runs > 0 ? pl->timed_runs : 1;
+    *prefill_ms_out = (float)(acc[0] / n);
+    *decode_ms_out = (float)(acc[1] / n);
+    *merge_ms_out = (float)(acc[2] / n);
+    *n_runs_out = pl->timed_runs;
+    return PS_OK;
 }
 
 ps_status ps_plan_status(ps_plan* pl, void* stream) {

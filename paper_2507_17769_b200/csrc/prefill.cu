@@ -290,8 +290,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                             p0 = (c0 + c < vis) ? p0 : 0.f;
                             p1 = (c0 + c + 1 < vis) ? p1 : 0.f;
                         }
-                        l += p0 + p1;
-                        packed[c >> 1] = pack_bf16(p0, p1);
+                        // sum the bf16-rounded weights PV multiplies: the output stays a convex mix of V rows
+                        const uint32_t pk = pack_bf16(p0, p1);
+                        l += bf16_lo(pk) + bf16_hi(pk);
+                        packed[c >> 1] = pk;
                     }
                     char* prow = smem + Cfg::kOffP + (c0 >> 6) * Cfg::kHalfBytes + t * 128;
 #pragma unroll
