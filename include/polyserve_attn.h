@@ -197,6 +197,39 @@ ps_status ps_attn_run(ps_plan *plan, const ps_kv *kv, const void *q_dev, const i
 ps_status ps_plan_status(ps_plan *plan, void *stream);
 
 /*
+ * ps_attn_run without a caller-provided workspace.  (The paper has no
+ * counterpart for this call; it exists for integration reasons only.)
+ *
+ * Some callers cannot hand the library device memory at the moment they need
+ * attention: a plug-in running inside a host engine that owns every byte of
+ * HBM and forbids cudaMalloc after start-up, a latency-critical loop where an
+ * allocation would stall the device, or a process whose memory budget is fixed
+ * when it loads.  For them the scratch that ps_attn_run takes as
+ * `workspace_dev` (the uploaded work list and the split-KV partial results
+ * passed from the decode / prefill kernels to the merge kernel) lives in a
+ * fixed array of PS_STATIC_WORKSPACE_BYTES inside the library's device image.
+ * Every GPU that loads the library keeps that array until the process exits.
+ *
+ * Arguments and results are those of ps_attn_run; inputs, outputs, pool and
+ * plan are still the caller's.  This call itself allocates nothing, on the
+ * host or on the device (the plan was allocated earlier by ps_attn_plan).
+ * A plan whose workspace need exceeds PS_STATIC_WORKSPACE_BYTES is refused
+ * with PS_ERR_WORKSPACE before anything is launched: use ps_attn_run, or
+ * smaller batches.
+ *
+ * The first call on each device looks up the array's device address (a
+ * runtime query made with that device current, as it must be at every call);
+ * make that first call before starting any stream capture.  All calls on a
+ * device share the one array and it keeps whatever the last call left there:
+ * each run rewrites the header words that must start at zero, but two runs
+ * that overlap on the GPU (different streams, or different plans in flight)
+ * would overwrite each other's work list and partials -- serialise them.
+ */
+#define PS_STATIC_WORKSPACE_BYTES (8u << 20)
+ps_status ps_attn_run_static(ps_plan *plan, const ps_kv *kv, const void *q_dev, const int32_t *block_table_dev,
+                             void *out_dev, float *lse_out_dev, void *stream);
+
+/*
  * Per-kernel timing of the next runs of this plan (the profile of section 4.5
  * split into its prefill-attention and decode-attention terms, section 3.4).
  * ps_plan_set_timing(plan, max_runs) makes each of the next max_runs calls of

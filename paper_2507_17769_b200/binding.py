@@ -63,7 +63,7 @@ class ps_grid_row(ctypes.Structure):
 
 EXPORTS = ["ps_kv_bytes", "ps_kv_alloc", "ps_kv_free", "ps_kv_write", "ps_kv_gather", "ps_kv_status", "ps_attn_plan",
            "ps_plan_free", "ps_plan_get_info", "ps_plan_get_items", "ps_attn_run", "ps_plan_status",
-           "ps_plan_set_timing", "ps_plan_get_timing", "ps_profile_grid",
+           "ps_plan_set_timing", "ps_plan_get_timing", "ps_profile_grid", "ps_attn_run_static",
            "ps_last_error", "ps_version"]
 
 _lib = None
@@ -94,6 +94,7 @@ def load() -> ctypes.CDLL:
     lib.ps_plan_get_items.argtypes = [_vp, _i32p, _i64, _i32p, _i64]
     lib.ps_attn_run.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
     lib.ps_plan_status.argtypes = [_vp, _vp]
+    lib.ps_attn_run_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
     lib.ps_plan_set_timing.argtypes = [_vp, _i32]
     fp = ctypes.POINTER(ctypes.c_float)
     lib.ps_plan_get_timing.argtypes = [_vp, _vp, fp, fp, fp, ctypes.POINTER(_i32)]
@@ -204,6 +205,20 @@ def ps_plan_get_items(plan):
 def ps_attn_run(plan, kv, q_dev, block_table_dev, out_dev, lse_out_dev, workspace_dev, workspace_bytes, stream=None):
     _check(load().ps_attn_run(plan, kv, _ptr(q_dev), _ptr(block_table_dev), _ptr(out_dev), _ptr(lse_out_dev),
                               _ptr(workspace_dev), workspace_bytes, _ptr(stream)))
+
+
+PS_STATIC_WORKSPACE_BYTES = 8 << 20
+
+
+def ps_attn_run_static(plan, kv, q_dev, block_table_dev, out_dev, lse_out_dev, stream=None):
+    """ps_attn_run on the library's built-in scratch array: no workspace argument, no allocation.
+
+    For callers that may not allocate device memory when they need attention.
+    Plans needing more than PS_STATIC_WORKSPACE_BYTES raise PS_ERR_WORKSPACE.
+    Calls on one device share the array: do not let two of them overlap on the GPU.
+    """
+    _check(load().ps_attn_run_static(plan, kv, _ptr(q_dev), _ptr(block_table_dev), _ptr(out_dev), _ptr(lse_out_dev),
+                                     _ptr(stream)))
 
 
 def ps_plan_status(plan, stream=None):

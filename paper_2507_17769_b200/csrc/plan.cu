@@ -452,3 +452,7 @@ ps_status ps_plan_status(ps_plan* pl, void* stream) {
 }
 
 }  // extern "C"
+
+namespace ps {
+size_t plan_workspace_bytes(const ps_plan* pl) { return pl ? pl->ws_bytes : 0; }
+}  // namespace ps
