@@ -162,7 +162,7 @@ ps_status ps_plan_get_info(const ps_plan *plan, ps_plan_info *info_out);
  * 8 int32: {request, kv_head, key_begin, key_end, q_token, n_tokens,
  * partial_slot, first_position}.  q_token is the packed index of the item's
  * first q token, n_tokens how many consecutive q tokens it covers (1 for
- * decode), partial_slot is -1 when the item writes final output, and
+ * decode, at most 256 / G for prefill), partial_slot is -1 when the item writes final output, and
  * first_position = prior + index of its first token in the chunk.  Either
  * output may be NULL; capacities are in items.
  */

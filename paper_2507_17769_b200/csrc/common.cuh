@@ -69,6 +69,9 @@ const KvPool& pool_of(const ps_kv* kv);
 // ---------------------------------------------------------------------------
 // device work list
 // ---------------------------------------------------------------------------
+// (token, head) rows one prefill item covers: two q tiles of 128 rows that share their K/V stream
+constexpr int kPrefillRowsPerItem = 256;
+
 constexpr int kStatusOk = 0, kStatusBounds = 1, kStatusTimeout = 2;
 
 struct WsHeader {         // 64 bytes at the start of the workspace
@@ -103,7 +106,7 @@ struct PrefillItem {
     int32_t key_begin;    // multiple of 128
     int32_t key_end;      // exclusive; <= first_pos + n_tok
     int32_t q_tok;        // packed index of the tile's first q token
-    int32_t n_tok;        // q tokens in the tile (<= 128 / G)
+    int32_t n_tok;        // q tokens in the item (<= 256 / G)
     int32_t part_slot;    // partial slot of (segment, token 0, head 0), or -1: write final output
     int32_t first_pos;    // absolute position of the tile's first q token (prior + index in chunk)
 };

@@ -19,7 +19,6 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 constexpr int kDecodeUnitsPerWarp = 2;  // dynamic-queue units per resident warp
 constexpr int kDecodeMinPages = 8;      // smallest decode unit (pages)
 constexpr int kPrefillKeyTile = 128;    // keys per tensor-core tile
-constexpr int kPrefillRows = 128;       // (token, head) rows per q tile
 
 }  // namespace ps
 
@@ -120,7 +119,7 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
 static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len, const std::vector<int32_t>& q_start,
                          const ps_plan_opts* opts, int64_t* n_slots) {
     const int Hkv = pl->shape.n_kv_heads, G = pl->shape.n_q_heads / Hkv;
-    const int tile_tok = kPrefillRows / G;
+    const int tile_tok = kPrefillRowsPerItem / G;
     struct Tile { int r, g, tok0, n_tok, first_pos, key_tiles; };
     std::vector<Tile> tiles;
     int64_t total_key_tiles = 0;

@@ -5,19 +5,25 @@
 // bound (section 3.4), so QK^T and PV run as tcgen05.mma with fp32
 // accumulators in tensor memory.
 //
-// One CTA works on one item = a q tile of 128 (token, head) rows that share a
-// kv head (the group's G heads of 128 / G consecutive tokens) x a key range.
-// Roles:
-//   warps 0-3  softmax: thread t owns row t (= TMEM lane t); reads S with
-//              tcgen05.ld, masks by the causal limit prior + i, keeps a
-//              running max with lazy rescaling of O, writes P (bf16) to shared
-//              memory in the operand layout, normalises and stores O at the end
-//   warp 4     producer: one 2 KB bulk async copy per (page, K|V, d half) into
-//              a 2-stage ring; the pool's page layout already is the
+// One CTA works on one item = up to two consecutive q tiles (A, B) of 128
+// (token, head) rows each -- the G heads that share a kv head x 128 / G
+// consecutive tokens -- over one key range.  Both tiles consume the same K and V
+// tiles from shared memory, and while one tile's softmax runs on the CUDA cores
+// the tensor core works for the other tile (ping-pong).
+//
+//   warps 0-3  softmax of tile A: thread t owns row t (= TMEM lane t); one
+//              tcgen05.ld pass over S, causal mask by prior + i, running max
+//              with lazy rescaling of O, P (bf16) stored back into the TMEM
+//              columns S occupied, O / l and the log-sum-exp at the end
+//   warps 4-7  the same for tile B
+//   warp 8     producer: one 2 KB bulk async copy per (page, K|V, d half) into
+//              2-stage K and V rings; the pool's page layout already is the
 //              128-byte-swizzled operand layout, so blocks are consumed in place
-//   warp 5     MMA issue: S[b] = Q K^T (8 x M128 N128 K16), O += P V
-//              (8 x M128 N=d K16), software-pipelined so QK^T of tile j+1
-//              overlaps the softmax of tile j; completion via tcgen05.commit
+//   warp 9     MMA issue: S_X = Q_X K^T (SS form, M128 N128 K16) and
+//              O_X += P_X V (A operand from TMEM, V as MN-major B operand,
+//              M128 N=d K16); completion signalled with tcgen05.commit
+//
+// TMEM columns: S_A 0..127, S_B 128..255, O_A 256.., O_B 384.. (512 allocated).
 // Every wait is bounded; on expiry the CTA sets the timeout status and drains.
 #include "common.cuh"
 
@@ -25,7 +31,9 @@ namespace ps {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kSoftmaxThreads = 256;
+constexpr int kThreads = kSoftmaxThreads + 64;
+constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr int kTileKeys = 128;
 constexpr int kRows = 128;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
@@ -51,6 +59,14 @@ __device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t a_desc, uint
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem desc]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -99,19 +115,17 @@ template <int D>
 struct PrefillCfg {
     static constexpr int kHalves = D / 64;
     static constexpr int kHalfBytes = kTileKeys * 128;          // [128 rows][128 B]
-    static constexpr int kQBytes = kHalves * kHalfBytes;         // Q tile
+    static constexpr int kQBytes = kHalves * kHalfBytes;         // one Q tile
     static constexpr int kKBytes = kHalves * kHalfBytes;         // one K stage
     static constexpr int kVBytes = kHalves * kHalfBytes;         // one V stage
-    static constexpr int kPBytes = 2 * kHalfBytes;               // P: two 64-key halves
     static constexpr int kStages = 2;
-    static constexpr int kOffQ = 0;
-    static constexpr int kOffK = kOffQ + kQBytes;
+    static constexpr int kOffQ = 0;                              // Q_A, Q_B
+    static constexpr int kOffK = kOffQ + 2 * kQBytes;
     static constexpr int kOffV = kOffK + kStages * kKBytes;
-    static constexpr int kOffP = kOffV + kStages * kVBytes;
-    static constexpr int kOffBar = kOffP + kPBytes;
+    static constexpr int kOffBar = kOffV + kStages * kVBytes;
     static constexpr int kSmemBytes = kOffBar + 256 + 1024;      // + alignment slack
     static constexpr int kTmemCols = 512;
-    static constexpr uint32_t kColS0 = 0, kColS1 = 128, kColO = 256;
+    static constexpr uint32_t kColS = 0, kColO = 256, kColTile = 128;  // tile X at + X * 128
 };
 
 struct PrefillParams {
@@ -131,9 +145,9 @@ struct PrefillParams {
     float scale_log2;
 };
 
-struct Bars {  // byte offsets from the barrier block
-    static constexpr int k_full = 0, k_empty = 16, v_full = 32, v_empty = 48, s_full = 64, p_ready = 80, o_done = 88;
-    static constexpr int tmem_slot = 96, item_slot = 100, abort_slot = 104;
+struct Bars {  // byte offsets from the barrier block; [2] = one per stage or per tile
+    static constexpr int k_full = 0, k_empty = 16, v_full = 32, v_empty = 48, s_full = 64, p_ready = 80, o_done = 96;
+    static constexpr int tmem_slot = 112, item_slot = 116, abort_slot = 120;
 };
 
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
@@ -144,7 +158,6 @@ __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, vol
     *abort_flag = 1;
     return false;
 }
-
 // warp-uniform result, so that the warp-collective instructions that follow stay converged
 __device__ __forceinline__ bool wait_all(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     return __all_sync(0xffffffffu, wait_or_abort(bar, parity, abort_flag));
@@ -169,9 +182,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
             mbar_init(bars + Bars::v_full + 8 * s, 1);
             mbar_init(bars + Bars::v_empty + 8 * s, 1);
             mbar_init(bars + Bars::s_full + 8 * s, 1);
+            mbar_init(bars + Bars::p_ready + 8 * s, kRows);
+            mbar_init(bars + Bars::o_done + 8 * s, 1);
         }
-        mbar_init(bars + Bars::p_ready, kRows);
-        mbar_init(bars + Bars::o_done, 1);
         mbar_fence_init();
         *s_abort = 0;
     }
@@ -184,9 +197,14 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
     tc_fence_after();
     const uint32_t tmem = (uint32_t)*s_tmem;
 
-    uint32_t tile_ctr = 0;  // key tiles processed by this CTA so far (every role counts the same)
+    // Phase counters; every role advances them identically.  Tile B's barriers only move in
+    // items that have a second q tile, so they are counted separately.
+    uint32_t tile_ctr = 0, tile_ctr_b = 0;  // key tiles processed so far (all items / items with a tile B)
+    uint32_t item_ctr = 0, item_ctr_b = 0;  // items processed (phase of the per-item o_done barriers)
     constexpr uint32_t kIdescQK = instr_desc(kTileKeys, false);
     constexpr uint32_t kIdescPV = instr_desc(D, true);
+    static_assert(kPrefillRowsPerItem == 2 * kRows, "the planner pairs two q tiles per item");
+    const int tile_tok = kRows / p.G;
 
     while (true) {
         if (threadIdx.x == 0) *s_item = atomicAdd(&p.hdr->prefill_next, 1);
@@ -197,173 +215,192 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
         if (item_idx >= p.n_items || *s_abort) break;
         const PrefillItem it = p.items[item_idx];
         const int n_tiles = (it.key_end - it.key_begin + kTileKeys - 1) / kTileKeys;
+        const bool has_b = it.n_tok > tile_tok;
 
-        // ---- Q tile -> shared memory (row t = token t / G, head t % G) ----
-        if (warp < 4) {
-            const int t = threadIdx.x;
-            const int i = t / p.G, hh = t % p.G;
+        // ---- Q tiles -> shared memory (tile X row t = token X * tile_tok + t / G, head t % G) ----
+        if (warp < 8) {
+            const int x = warp >> 2, t = threadIdx.x & 127;
+            const int i = x * tile_tok + t / p.G, hh = t % p.G;
             const bool valid = i < it.n_tok;
             const uint4* src = reinterpret_cast<const uint4*>(
                 p.q + ((int64_t)(it.q_tok + (valid ? i : 0)) * p.Hq + it.kv_head * p.G + hh) * D);
+            char* qdst = smem + Cfg::kOffQ + x * Cfg::kQBytes + t * 128;
 #pragma unroll
             for (int U = 0; U < D / 8; ++U) {
                 const uint4 v = valid ? __ldg(src + U) : make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4*>(smem + Cfg::kOffQ + (U >> 3) * Cfg::kHalfBytes + t * 128 + (((U & 7) ^ (t & 7)) << 4)) = v;
+                *reinterpret_cast<uint4*>(qdst + (U >> 3) * Cfg::kHalfBytes + (((U & 7) ^ (t & 7)) << 4)) = v;
             }
             fence_proxy_async_smem();
         }
         __syncthreads();
 
-        if (warp < 4) {
-            // =========================== softmax ===========================
-            const int t = threadIdx.x;
-            const int i = t / p.G;
-            const int limit = it.first_pos + i;  // last visible key of this row
-            const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-            float m = -INFINITY, l = 0.f;
-            bool ok = true;
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const uint32_t tc = tile_ctr + j;
-                const uint32_t b = tc & 1;
-                ok = wait_all(bars + Bars::s_full + 8 * b, (tc >> 1) & 1, s_abort);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t s_addr = tmem + lane_addr + (b ? Cfg::kColS1 : Cfg::kColS0);
-                const int tile_base = it.key_begin + j * kTileKeys;
-                const bool need_mask = (tile_base + kTileKeys - 1 > it.first_pos) || (tile_base + kTileKeys > it.key_end);
-                const int vis = min(limit + 1, it.key_end) - tile_base;  // columns [0, vis) are visible to this row
-
-                // pass 1: row max of the raw scores
-                float mx = -INFINITY;
-#pragma unroll 1
-                for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(s_addr + c0, v);
-                    tmem_wait_ld();
-                    if (need_mask) {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) mx = (c0 + c < vis) ? fmaxf(mx, __uint_as_float(v[c])) : mx;
-                    } else {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) mx = fmaxf(mx, __uint_as_float(v[c]));
-                    }
-                }
-                const float mx_s = mx * p.scale_log2;
-                float m_new = m;
-                if (mx_s > m + kRescaleThreshold || (m == -INFINITY && mx_s > -INFINITY)) m_new = mx_s;
-                const float alpha = (m_new == m) ? 1.f : fast_exp2(m - m_new);
-
-                if (j > 0) {
-                    // PV of the previous tile must be done before P is overwritten or O rescaled
-                    ok = wait_all(bars + Bars::o_done, (tc - 1) & 1, s_abort);
+        if (warp < 8) {
+            // =========================== softmax of tile x ===========================
+            const int x = warp >> 2, t = threadIdx.x & 127;
+            if (x == 0 || has_b) {
+                const int i = x * tile_tok + t / p.G;
+                const int limit = it.first_pos + i;  // last visible key of this row
+                const int tile_first_pos = it.first_pos + x * tile_tok;
+                const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+                const uint32_t s_addr = tmem + lane_addr + Cfg::kColS + x * Cfg::kColTile;
+                const uint32_t o_addr = tmem + lane_addr + Cfg::kColO + x * Cfg::kColTile;
+                float m = -INFINITY, l = 0.f;
+                bool ok = true;
+                for (int j = 0; j < n_tiles && ok; ++j) {
+                    const uint32_t tc = tile_ctr + j;                          // K/V stage phase
+                    const uint32_t tcx = (x ? tile_ctr_b : tile_ctr) + j;     // phase of this tile's own barriers
+                    ok = wait_all(bars + Bars::s_full + 8 * x, tcx & 1, s_abort);
                     if (!ok) break;
                     tc_fence_after();
-                    if (__any_sync(0xffffffffu, m_new != m)) {
+                    const int tile_base = it.key_begin + j * kTileKeys;
+                    const bool need_mask = (tile_base + kTileKeys - 1 > tile_first_pos) || (tile_base + kTileKeys > it.key_end);
+                    const int vis = min(limit + 1, it.key_end) - tile_base;  // columns [0, vis) are visible to this row
+
+                    uint32_t sv[4][32];
+                    tmem_ld32(s_addr + 0, sv[0]);
+                    tmem_ld32(s_addr + 32, sv[1]);
+                    tmem_ld32(s_addr + 64, sv[2]);
+                    tmem_ld32(s_addr + 96, sv[3]);
+                    tmem_wait_ld();
+
+                    // row max of the raw scores, four independent chains
+                    float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                    if (need_mask) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4) {
+                                const int col = q * 32 + c;
+                                mx0 = (col < vis) ? fmaxf(mx0, __uint_as_float(sv[q][c])) : mx0;
+                                mx1 = (col + 1 < vis) ? fmaxf(mx1, __uint_as_float(sv[q][c + 1])) : mx1;
+                                mx2 = (col + 2 < vis) ? fmaxf(mx2, __uint_as_float(sv[q][c + 2])) : mx2;
+                                mx3 = (col + 3 < vis) ? fmaxf(mx3, __uint_as_float(sv[q][c + 3])) : mx3;
+                            }
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                            for (int c = 0; c < 32; c += 4) {
+                                mx0 = fmaxf(mx0, __uint_as_float(sv[q][c]));
+                                mx1 = fmaxf(mx1, __uint_as_float(sv[q][c + 1]));
+                                mx2 = fmaxf(mx2, __uint_as_float(sv[q][c + 2]));
+                                mx3 = fmaxf(mx3, __uint_as_float(sv[q][c + 3]));
+                            }
+                    }
+                    const float mx_s = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+                    float m_new = m;
+                    if (mx_s > m + kRescaleThreshold) m_new = mx_s;  // also the first finite max (m = -inf)
+                    const float alpha = (m_new == m) ? 1.f : fast_exp2(m - m_new);
+
+                    // O_x holds tiles 0..j-1 (the commit that raised s_full came after PV_x(j-1))
+                    if (j > 0 && __any_sync(0xffffffffu, m_new != m)) {
 #pragma unroll 1
                         for (int c0 = 0; c0 < D; c0 += 32) {
                             uint32_t v[32];
-                            tmem_ld32(tmem + lane_addr + Cfg::kColO + c0, v);
+                            tmem_ld32(o_addr + c0, v);
                             tmem_wait_ld();
 #pragma unroll
                             for (int c = 0; c < 32; ++c) v[c] = __float_as_uint(__uint_as_float(v[c]) * alpha);
-                            tmem_st32(tmem + lane_addr + Cfg::kColO + c0, v);
+                            tmem_st32(o_addr + c0, v);
                         }
                         tmem_wait_st();
                     }
-                }
-                l *= alpha;
-                m = m_new;
-                const float m_sub = (m == -INFINITY) ? 0.f : m;
+                    l *= alpha;
+                    m = m_new;
+                    const float m_sub = (m == -INFINITY) ? 0.f : m;
 
-                // pass 2: P = exp2(scale * s - m), bf16, into the A-operand layout
-#pragma unroll 1
-                for (int c0 = 0; c0 < kTileKeys; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(s_addr + c0, v);
-                    tmem_wait_ld();
-                    uint32_t packed[16];
+                    // P = exp2(scale * s - m) as bf16 pairs, written over S's first 64 columns
+                    float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-                    for (int c = 0; c < 32; c += 2) {
-                        float p0 = fast_exp2(fmaf(__uint_as_float(v[c]), p.scale_log2, -m_sub));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(v[c + 1]), p.scale_log2, -m_sub));
-                        if (need_mask) {
-                            p0 = (c0 + c < vis) ? p0 : 0.f;
-                            p1 = (c0 + c + 1 < vis) ? p1 : 0.f;
+                    for (int hhalf = 0; hhalf < 2; ++hhalf) {
+                        uint32_t packed[32];
+#pragma unroll
+                        for (int qq = 0; qq < 2; ++qq) {
+                            const int q = hhalf * 2 + qq;
+#pragma unroll
+                            for (int c = 0; c < 32; c += 2) {
+                                float p0 = fast_exp2(fmaf(__uint_as_float(sv[q][c]), p.scale_log2, -m_sub));
+                                float p1 = fast_exp2(fmaf(__uint_as_float(sv[q][c + 1]), p.scale_log2, -m_sub));
+                                if (need_mask) {
+                                    p0 = (q * 32 + c < vis) ? p0 : 0.f;
+                                    p1 = (q * 32 + c + 1 < vis) ? p1 : 0.f;
+                                }
+                                // sum the bf16-rounded weights PV multiplies: the output stays a convex mix of V rows
+                                const uint32_t pk = pack_bf16(p0, p1);
+                                l0 += bf16_lo(pk);
+                                l1 += bf16_hi(pk);
+                                packed[qq * 16 + (c >> 1)] = pk;
+                            }
                         }
-                        // sum the bf16-rounded weights PV multiplies: the output stays a convex mix of V rows
-                        const uint32_t pk = pack_bf16(p0, p1);
-                        l += bf16_lo(pk) + bf16_hi(pk);
-                        packed[c >> 1] = pk;
+                        tmem_st32(s_addr + hhalf * 32, packed);
                     }
-                    char* prow = smem + Cfg::kOffP + (c0 >> 6) * Cfg::kHalfBytes + t * 128;
+                    l += l0 + l1;
+                    tmem_wait_st();
+
+                    // keys at or past key_end: their V rows may be stale or poisoned; zero them so 0 * V = 0
+                    const int n_keys = it.key_end - tile_base;
+                    if (x == 0 && n_keys < kTileKeys) {
+                        const uint32_t s = tc & 1;
+                        ok = wait_all(bars + Bars::v_full + 8 * s, (tc >> 1) & 1, s_abort);
+                        if (!ok) break;
+                        if (t >= n_keys) {
+                            char* vrow = smem + Cfg::kOffV + s * Cfg::kVBytes + t * 128;
 #pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const int unit = ((c0 & 63) >> 3) + u;
-                        *reinterpret_cast<uint4*>(prow + ((unit ^ (t & 7)) << 4)) =
-                            make_uint4(packed[4 * u], packed[4 * u + 1], packed[4 * u + 2], packed[4 * u + 3]);
+                            for (int h = 0; h < Cfg::kHalves; ++h)
+#pragma unroll
+                                for (int u = 0; u < 8; ++u)
+                                    *reinterpret_cast<uint4*>(vrow + h * Cfg::kHalfBytes + u * 16) = make_uint4(0, 0, 0, 0);
+                        }
+                        fence_proxy_async_smem();
                     }
+                    tc_fence_before();
+                    mbar_arrive(bars + Bars::p_ready + 8 * x);
                 }
-                // keys at or past key_end: their V rows may be stale or poisoned; zero them so 0 * V = 0
-                const int n_keys = it.key_end - tile_base;
-                if (n_keys < kTileKeys) {
-                    ok = wait_all(bars + Bars::v_full + 8 * b, (tc >> 1) & 1, s_abort);
-                    if (!ok) break;
-                    if (t >= n_keys) {
-                        char* vrow = smem + Cfg::kOffV + b * Cfg::kVBytes + t * 128;
+                // ---- epilogue: O / l ----
+                if (ok) ok = wait_all(bars + Bars::o_done + 8 * x, (x ? item_ctr_b : item_ctr) & 1, s_abort);
+                if (ok) {
+                    tc_fence_after();
+                    const float inv = l > 0.f ? 1.f / l : 0.f;
+                    const float lse_v = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
+                    const bool valid = i < it.n_tok;
+                    const int hh = t % p.G;
+                    const int64_t orow = (int64_t)(it.q_tok + i) * p.Hq + it.kv_head * p.G + hh;
+                    const int64_t prow = (int64_t)it.part_slot + (int64_t)i * p.G + hh;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < D; c0 += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(o_addr + c0, v);
+                        tmem_wait_ld();
+                        if (!valid) continue;
+                        if (it.part_slot < 0) {
+                            uint4* dst = reinterpret_cast<uint4*>(p.out + orow * D + c0);
 #pragma unroll
-                        for (int h = 0; h < Cfg::kHalves; ++h)
+                            for (int u = 0; u < 4; ++u) {
+                                uint4 w;
+                                w.x = pack_bf16(__uint_as_float(v[8 * u + 0]) * inv, __uint_as_float(v[8 * u + 1]) * inv);
+                                w.y = pack_bf16(__uint_as_float(v[8 * u + 2]) * inv, __uint_as_float(v[8 * u + 3]) * inv);
+                                w.z = pack_bf16(__uint_as_float(v[8 * u + 4]) * inv, __uint_as_float(v[8 * u + 5]) * inv);
+                                w.w = pack_bf16(__uint_as_float(v[8 * u + 6]) * inv, __uint_as_float(v[8 * u + 7]) * inv);
+                                dst[u] = w;
+                            }
+                        } else {
+                            float4* dst = reinterpret_cast<float4*>(p.part_o + prow * D + c0);
 #pragma unroll
                             for (int u = 0; u < 8; ++u)
-                                *reinterpret_cast<uint4*>(vrow + h * Cfg::kHalfBytes + u * 16) = make_uint4(0, 0, 0, 0);
-                    }
-                }
-                fence_proxy_async_smem();
-                tc_fence_before();
-                mbar_arrive(bars + Bars::p_ready);
-            }
-            // ---- epilogue: O / l ----
-            if (ok) ok = wait_all(bars + Bars::o_done, (tile_ctr + n_tiles - 1) & 1, s_abort);
-            if (ok) {
-                tc_fence_after();
-                const float inv = l > 0.f ? 1.f / l : 0.f;
-                const float lse_v = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
-                const bool valid = i < it.n_tok;
-                const int hh = t % p.G;
-                const int64_t orow = (int64_t)(it.q_tok + i) * p.Hq + it.kv_head * p.G + hh;
-#pragma unroll 1
-                for (int c0 = 0; c0 < D; c0 += 32) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem + lane_addr + Cfg::kColO + c0, v);
-                    tmem_wait_ld();
-                    if (!valid) continue;
-                    if (it.part_slot < 0) {
-                        uint4* dst = reinterpret_cast<uint4*>(p.out + orow * D + c0);
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            uint4 w;
-                            w.x = pack_bf16(__uint_as_float(v[8 * u + 0]) * inv, __uint_as_float(v[8 * u + 1]) * inv);
-                            w.y = pack_bf16(__uint_as_float(v[8 * u + 2]) * inv, __uint_as_float(v[8 * u + 3]) * inv);
-                            w.z = pack_bf16(__uint_as_float(v[8 * u + 4]) * inv, __uint_as_float(v[8 * u + 5]) * inv);
-                            w.w = pack_bf16(__uint_as_float(v[8 * u + 6]) * inv, __uint_as_float(v[8 * u + 7]) * inv);
-                            dst[u] = w;
+                                dst[u] = make_float4(__uint_as_float(v[4 * u]) * inv, __uint_as_float(v[4 * u + 1]) * inv,
+                                                     __uint_as_float(v[4 * u + 2]) * inv, __uint_as_float(v[4 * u + 3]) * inv);
                         }
-                    } else {
-                        float4* dst = reinterpret_cast<float4*>(p.part_o + ((int64_t)it.part_slot + t) * D + c0);
-#pragma unroll
-                        for (int u = 0; u < 8; ++u)
-                            dst[u] = make_float4(__uint_as_float(v[4 * u]) * inv, __uint_as_float(v[4 * u + 1]) * inv,
-                                                 __uint_as_float(v[4 * u + 2]) * inv, __uint_as_float(v[4 * u + 3]) * inv);
                     }
-                }
-                if (valid) {
-                    if (it.part_slot < 0) {
-                        if (p.lse) p.lse[orow] = lse_v;
-                    } else {
-                        p.part_lse[it.part_slot + t] = lse_v;
+                    if (valid) {
+                        if (it.part_slot < 0) {
+                            if (p.lse) p.lse[orow] = lse_v;
+                        } else {
+                            p.part_lse[prow] = lse_v;
+                        }
                     }
                 }
             }
-        } else if (warp == 4) {
+        } else if (warp == kProducerWarp) {
             // =========================== producer ===========================
             const int pg = lane >> 2, which = lane & 3;  // page in tile; 0/1 = K half 0/1, 2/3 = V half 0/1
             const int32_t* bt = p.block_table + (int64_t)it.req * p.max_pages + it.key_begin / kPage;
@@ -374,7 +411,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                 const uint32_t s = tc & 1, par = (tc >> 1) & 1;
                 const int n_keys = min(kTileKeys, it.key_end - (it.key_begin + j * kTileKeys));
                 const int n_pages = (n_keys + kPage - 1) / kPage;
-                int page = (lane < n_pages) ? __ldg(bt + j * 8 + lane) : 0;
+                const int page = (lane < n_pages) ? __ldg(bt + j * 8 + lane) : 0;
                 const bool in_range = (uint32_t)page < (uint64_t)p.num_pages;
                 const uint32_t good = __ballot_sync(0xffffffffu, lane < n_pages && in_range);
                 if (__popc(good) != n_pages && lane == 0) atomicOr(&p.hdr->status, kStatusBounds);
@@ -402,50 +439,66 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
         } else {
             // =========================== MMA issue ===========================
             bool ok = true;
-            auto issue_qk = [&](int j) {
+            const int n_x = has_b ? 2 : 1;
+            // S_x(j) = Q_x K(j)^T; the last tile to read K stage s releases it
+            auto issue_qk = [&](int j, int x) {
                 const uint32_t tc = tile_ctr + j;
                 const uint32_t s = tc & 1;
-                ok = wait_all(bars + Bars::k_full + 8 * s, (tc >> 1) & 1, s_abort);
-                if (!ok) return;
-                tc_fence_after();
+                if (x == 0) {
+                    ok = wait_all(bars + Bars::k_full + 8 * s, (tc >> 1) & 1, s_abort);
+                    if (!ok) return;
+                    tc_fence_after();
+                }
                 if (lane == 0) {
-                    const uint32_t d_addr = tmem + (s ? Cfg::kColS1 : Cfg::kColS0);
+                    const uint32_t d_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
                         const uint32_t off = (kk >> 2) * Cfg::kHalfBytes + (kk & 3) * 32;
-                        tc_mma_ss(d_addr, smem_desc(sbase + Cfg::kOffQ + off, 16, 1024),
+                        tc_mma_ss(d_addr, smem_desc(sbase + Cfg::kOffQ + x * Cfg::kQBytes + off, 16, 1024),
                                   smem_desc(sbase + Cfg::kOffK + s * Cfg::kKBytes + off, 16, 1024), kIdescQK, kk > 0);
                     }
-                    tc_commit(bars + Bars::s_full + 8 * s);
-                    tc_commit(bars + Bars::k_empty + 8 * s);
+                    tc_commit(bars + Bars::s_full + 8 * x);
+                    if (x == n_x - 1) tc_commit(bars + Bars::k_empty + 8 * s);
                 }
                 __syncwarp();
             };
-            issue_qk(0);
+            for (int x = 0; x < n_x && ok; ++x) issue_qk(0, x);
             for (int j = 0; j < n_tiles && ok; ++j) {
-                if (j + 1 < n_tiles) issue_qk(j + 1);
-                if (!ok) break;
                 const uint32_t tc = tile_ctr + j;
                 const uint32_t s = tc & 1;
-                ok = wait_all(bars + Bars::p_ready, tc & 1, s_abort);
-                if (!ok) break;
-                ok = wait_all(bars + Bars::v_full + 8 * s, (tc >> 1) & 1, s_abort);
-                if (!ok) break;
-                tc_fence_after();
-                if (lane == 0) {
-#pragma unroll
-                    for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-                        const uint64_t a = smem_desc(sbase + Cfg::kOffP + (kk >> 2) * Cfg::kHalfBytes + (kk & 3) * 32, 16, 1024);
-                        const uint64_t bdesc = smem_desc(sbase + Cfg::kOffV + s * Cfg::kVBytes + kk * 2048, Cfg::kHalfBytes, 1024);
-                        tc_mma_ss(tmem + Cfg::kColO, a, bdesc, kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                for (int x = 0; x < n_x && ok; ++x) {
+                    ok = wait_all(bars + Bars::p_ready + 8 * x, ((x ? tile_ctr_b : tile_ctr) + j) & 1, s_abort);
+                    if (!ok) break;
+                    if (x == 0) {
+                        ok = wait_all(bars + Bars::v_full + 8 * s, (tc >> 1) & 1, s_abort);
+                        if (!ok) break;
                     }
-                    tc_commit(bars + Bars::o_done);
-                    tc_commit(bars + Bars::v_empty + 8 * s);
+                    tc_fence_after();
+                    if (lane == 0) {
+                        // O_x += P_x V(j): P_x sits in S_x's first 64 columns, two bf16 per column
+                        const uint32_t a_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
+                        const uint32_t d_addr = tmem + Cfg::kColO + x * Cfg::kColTile;
+#pragma unroll
+                        for (int kk = 0; kk < kTileKeys / 16; ++kk) {
+                            const uint64_t bdesc = smem_desc(sbase + Cfg::kOffV + s * Cfg::kVBytes + kk * 2048, Cfg::kHalfBytes, 1024);
+                            tc_mma_ts(d_addr, a_addr + kk * 8, bdesc, kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                        }
+                        if (j == n_tiles - 1) tc_commit(bars + Bars::o_done + 8 * x);
+                        if (x == n_x - 1) tc_commit(bars + Bars::v_empty + 8 * s);
+                    }
+                    __syncwarp();
+                    // the tensor pipe runs this thread's MMAs in issue order, so S_x may be
+                    // overwritten by the next QK^T right behind the PV that reads P_x
+                    if (j + 1 < n_tiles) issue_qk(j + 1, x);
                 }
-                __syncwarp();
             }
         }
         tile_ctr += n_tiles;
+        ++item_ctr;
+        if (has_b) {
+            tile_ctr_b += n_tiles;
+            ++item_ctr_b;
+        }
     }
 
     // after an abort: flag the run and give copies in flight a bounded time to land

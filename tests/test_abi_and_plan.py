@@ -83,14 +83,14 @@ def coverage_check(batch, plan):
         r, g, k0, k1, qt, nt, slot, fp = it.tolist()
         assert batch.q_len[r] > 1 and k0 % 128 == 0 and k0 < k1
         tok0 = qt - q_start[r]
-        assert fp == batch.prior[r] + tok0 and 1 <= nt <= 128 // G and tok0 % (128 // G) == 0
+        assert fp == batch.prior[r] + tok0 and 1 <= nt <= 256 // G and tok0 % (256 // G) == 0
         assert k1 <= fp + nt
         tiles.setdefault((r, g, tok0, nt), []).append((k0, k1, slot))
     for r in range(batch.n):
         c = int(batch.q_len[r])
         if c <= 1:
             continue
-        tt = 128 // G
+        tt = 256 // G
         for g in range(s.n_kv_heads):
             covered = 0
             for tok0 in range(0, c, tt):
