@@ -32,7 +32,11 @@ namespace ps {
 namespace {
 
 constexpr int kSoftmaxThreads = 256;
-constexpr int kThreads = kSoftmaxThreads + 64;
+// Three warpgroups: two of softmax warps and one holding the producer and MMA warps (its
+// other two warps only take part in the CTA-wide barriers).  Registers are re-split after
+// start-up: 384 threads x 168 at launch = 2 x 128 x 200 + 128 x 104.
+constexpr int kThreads = kSoftmaxThreads + 128;
+constexpr int kRegsSoftmax = 200, kRegsOther = 104;
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr int kTileKeys = 128;
 constexpr int kRows = 128;
@@ -91,6 +95,30 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
           "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
           "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
+}
+// 3-input max and packed fp32 pairs (two lanes per 64-bit register)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -206,44 +234,62 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
     static_assert(kPrefillRowsPerItem == 2 * kRows, "the planner pairs two q tiles per item");
     const int tile_tok = kRows / p.G;
 
-    while (true) {
+    // Every role runs this at the top of each item; two CTA-wide barriers per item (after the
+    // item fetch, after the Q tiles are in shared memory) are executed by all 12 warps.
+    PrefillItem it;
+    int n_tiles = 0;
+    bool has_b = false;
+    auto next_item = [&]() -> bool {
         if (threadIdx.x == 0) *s_item = atomicAdd(&p.hdr->prefill_next, 1);
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
         const int item_idx = *s_item;
-        if (item_idx >= p.n_items || *s_abort) break;
-        const PrefillItem it = p.items[item_idx];
-        const int n_tiles = (it.key_end - it.key_begin + kTileKeys - 1) / kTileKeys;
-        const bool has_b = it.n_tok > tile_tok;
-
-        // ---- Q tiles -> shared memory (tile X row t = token X * tile_tok + t / G, head t % G) ----
-        if (warp < 8) {
-            const int x = warp >> 2, t = threadIdx.x & 127;
-            const int i = x * tile_tok + t / p.G, hh = t % p.G;
-            const bool valid = i < it.n_tok;
-            const uint4* src = reinterpret_cast<const uint4*>(
-                p.q + ((int64_t)(it.q_tok + (valid ? i : 0)) * p.Hq + it.kv_head * p.G + hh) * D);
-            char* qdst = smem + Cfg::kOffQ + x * Cfg::kQBytes + t * 128;
-#pragma unroll
-            for (int U = 0; U < D / 8; ++U) {
-                const uint4 v = valid ? __ldg(src + U) : make_uint4(0, 0, 0, 0);
-                *reinterpret_cast<uint4*>(qdst + (U >> 3) * Cfg::kHalfBytes + (((U & 7) ^ (t & 7)) << 4)) = v;
-            }
-            fence_proxy_async_smem();
+        if (item_idx >= p.n_items || *s_abort) return false;
+        it = p.items[item_idx];
+        n_tiles = (it.key_end - it.key_begin + kTileKeys - 1) / kTileKeys;
+        has_b = it.n_tok > tile_tok;
+        return true;
+    };
+    auto advance = [&]() {
+        tile_ctr += n_tiles;
+        ++item_ctr;
+        if (has_b) {
+            tile_ctr_b += n_tiles;
+            ++item_ctr_b;
         }
-        __syncthreads();
+    };
 
-        if (warp < 8) {
-            // =========================== softmax of tile x ===========================
-            const int x = warp >> 2, t = threadIdx.x & 127;
+    if (warp < 8) {
+        // ====================================================================
+        // softmax warpgroups: tile x = warp / 4, row t = thread within the group
+        // ====================================================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsSoftmax));
+        const int x = warp >> 2, t = threadIdx.x & 127;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t s_addr = tmem + lane_addr + Cfg::kColS + x * Cfg::kColTile;
+        const uint32_t o_addr = tmem + lane_addr + Cfg::kColO + x * Cfg::kColTile;
+        const int hh = t % p.G;
+        while (next_item()) {
+            // ---- Q tile x -> shared memory (row t = token x * tile_tok + t / G, head t % G) ----
+            const int i = x * tile_tok + t / p.G;
+            const bool valid = i < it.n_tok;
+            {
+                const uint4* src = reinterpret_cast<const uint4*>(
+                    p.q + ((int64_t)(it.q_tok + (valid ? i : 0)) * p.Hq + it.kv_head * p.G + hh) * D);
+                char* qdst = smem + Cfg::kOffQ + x * Cfg::kQBytes + t * 128;
+#pragma unroll
+                for (int U = 0; U < D / 8; ++U) {
+                    const uint4 v = valid ? __ldg(src + U) : make_uint4(0, 0, 0, 0);
+                    *reinterpret_cast<uint4*>(qdst + (U >> 3) * Cfg::kHalfBytes + (((U & 7) ^ (t & 7)) << 4)) = v;
+                }
+                fence_proxy_async_smem();
+            }
+            __syncthreads();
+
             if (x == 0 || has_b) {
-                const int i = x * tile_tok + t / p.G;
                 const int limit = it.first_pos + i;  // last visible key of this row
                 const int tile_first_pos = it.first_pos + x * tile_tok;
-                const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-                const uint32_t s_addr = tmem + lane_addr + Cfg::kColS + x * Cfg::kColTile;
-                const uint32_t o_addr = tmem + lane_addr + Cfg::kColO + x * Cfg::kColTile;
                 float m = -INFINITY, l = 0.f;
                 bool ok = true;
                 for (int j = 0; j < n_tiles && ok; ++j) {
@@ -280,11 +326,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
 #pragma unroll
-                            for (int c = 0; c < 32; c += 4) {
-                                mx0 = fmaxf(mx0, __uint_as_float(sv[q][c]));
-                                mx1 = fmaxf(mx1, __uint_as_float(sv[q][c + 1]));
-                                mx2 = fmaxf(mx2, __uint_as_float(sv[q][c + 2]));
-                                mx3 = fmaxf(mx3, __uint_as_float(sv[q][c + 3]));
+                            for (int c = 0; c < 32; c += 8) {
+                                mx0 = max3(mx0, __uint_as_float(sv[q][c]), __uint_as_float(sv[q][c + 1]));
+                                mx1 = max3(mx1, __uint_as_float(sv[q][c + 2]), __uint_as_float(sv[q][c + 3]));
+                                mx2 = max3(mx2, __uint_as_float(sv[q][c + 4]), __uint_as_float(sv[q][c + 5]));
+                                mx3 = max3(mx3, __uint_as_float(sv[q][c + 6]), __uint_as_float(sv[q][c + 7]));
                             }
                     }
                     const float mx_s = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
@@ -311,28 +357,61 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
 
                     // P = exp2(scale * s - m) as bf16 pairs, written over S's first 64 columns
                     float l0 = 0.f, l1 = 0.f;
+                    if (need_mask) {
+                        // Diagonal and ragged tiles (the only tiles of rows with few visible keys): mask by
+                        // select, and sum the bf16-rounded weights that PV multiplies, so that the output
+                        // of a row with a handful of keys stays an exact convex mix of V rows.
 #pragma unroll
-                    for (int hhalf = 0; hhalf < 2; ++hhalf) {
-                        uint32_t packed[32];
+                        for (int hhalf = 0; hhalf < 2; ++hhalf) {
+                            uint32_t packed[32];
 #pragma unroll
-                        for (int qq = 0; qq < 2; ++qq) {
-                            const int q = hhalf * 2 + qq;
+                            for (int qq = 0; qq < 2; ++qq) {
+                                const int q = hhalf * 2 + qq;
 #pragma unroll
-                            for (int c = 0; c < 32; c += 2) {
-                                float p0 = fast_exp2(fmaf(__uint_as_float(sv[q][c]), p.scale_log2, -m_sub));
-                                float p1 = fast_exp2(fmaf(__uint_as_float(sv[q][c + 1]), p.scale_log2, -m_sub));
-                                if (need_mask) {
+                                for (int c = 0; c < 32; c += 2) {
+                                    float p0 = fast_exp2(fmaf(__uint_as_float(sv[q][c]), p.scale_log2, -m_sub));
+                                    float p1 = fast_exp2(fmaf(__uint_as_float(sv[q][c + 1]), p.scale_log2, -m_sub));
                                     p0 = (q * 32 + c < vis) ? p0 : 0.f;
                                     p1 = (q * 32 + c + 1 < vis) ? p1 : 0.f;
+                                    const uint32_t pk = pack_bf16(p0, p1);
+                                    l0 += bf16_lo(pk);
+                                    l1 += bf16_hi(pk);
+                                    packed[qq * 16 + (c >> 1)] = pk;
                                 }
-                                // sum the bf16-rounded weights PV multiplies: the output stays a convex mix of V rows
-                                const uint32_t pk = pack_bf16(p0, p1);
-                                l0 += bf16_lo(pk);
-                                l1 += bf16_hi(pk);
-                                packed[qq * 16 + (c >> 1)] = pk;
                             }
+                            tmem_st32(s_addr + hhalf * 32, packed);
                         }
-                        tmem_st32(s_addr + hhalf * 32, packed);
+                    } else {
+                        // Interior tiles: two scores per instruction (packed fp32 FMA and add); four sum chains.
+                        const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(-m_sub, -m_sub);
+                        uint64_t ls0 = 0ull, ls1 = 0ull;
+#pragma unroll
+                        for (int hhalf = 0; hhalf < 2; ++hhalf) {
+                            uint32_t packed[32];
+#pragma unroll
+                            for (int qq = 0; qq < 2; ++qq) {
+                                const int q = hhalf * 2 + qq;
+#pragma unroll
+                                for (int c = 0; c < 32; c += 4) {
+                                    const uint64_t x01 = fma2(pack2(__uint_as_float(sv[q][c]), __uint_as_float(sv[q][c + 1])), sc2, nm2);
+                                    const uint64_t x23 = fma2(pack2(__uint_as_float(sv[q][c + 2]), __uint_as_float(sv[q][c + 3])), sc2, nm2);
+                                    float x0, x1, x2, x3;
+                                    unpack2(x01, x0, x1);
+                                    unpack2(x23, x2, x3);
+                                    const float e0 = fast_exp2(x0), e1 = fast_exp2(x1), e2 = fast_exp2(x2), e3 = fast_exp2(x3);
+                                    ls0 = add2(ls0, pack2(e0, e1));
+                                    ls1 = add2(ls1, pack2(e2, e3));
+                                    packed[qq * 16 + (c >> 1)] = pack_bf16(e0, e1);
+                                    packed[qq * 16 + (c >> 1) + 1] = pack_bf16(e2, e3);
+                                }
+                            }
+                            tmem_st32(s_addr + hhalf * 32, packed);
+                        }
+                        float a0, a1, a2, a3;
+                        unpack2(ls0, a0, a1);
+                        unpack2(ls1, a2, a3);
+                        l0 = a0 + a2;
+                        l1 = a1 + a3;
                     }
                     l += l0 + l1;
                     tmem_wait_st();
@@ -362,8 +441,6 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                     tc_fence_after();
                     const float inv = l > 0.f ? 1.f / l : 0.f;
                     const float lse_v = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
-                    const bool valid = i < it.n_tok;
-                    const int hh = t % p.G;
                     const int64_t orow = (int64_t)(it.q_tok + i) * p.Hq + it.kv_head * p.G + hh;
                     const int64_t prow = (int64_t)it.part_slot + (int64_t)i * p.G + hh;
 #pragma unroll 1
@@ -400,104 +477,123 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                     }
                 }
             }
-        } else if (warp == kProducerWarp) {
-            // =========================== producer ===========================
+            advance();
+        }
+    } else {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
+        if (warp == kProducerWarp) {
+            // ================================================================
+            // producer
+            // ================================================================
             const int pg = lane >> 2, which = lane & 3;  // page in tile; 0/1 = K half 0/1, 2/3 = V half 0/1
-            const int32_t* bt = p.block_table + (int64_t)it.req * p.max_pages + it.key_begin / kPage;
             constexpr uint32_t kPieceBytes = kPage * 128;  // 16 tokens x 64 elements
-            bool ok = true;
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const uint32_t tc = tile_ctr + j;
-                const uint32_t s = tc & 1, par = (tc >> 1) & 1;
-                const int n_keys = min(kTileKeys, it.key_end - (it.key_begin + j * kTileKeys));
-                const int n_pages = (n_keys + kPage - 1) / kPage;
-                const int page = (lane < n_pages) ? __ldg(bt + j * 8 + lane) : 0;
-                const bool in_range = (uint32_t)page < (uint64_t)p.num_pages;
-                const uint32_t good = __ballot_sync(0xffffffffu, lane < n_pages && in_range);
-                if (__popc(good) != n_pages && lane == 0) atomicOr(&p.hdr->status, kStatusBounds);
-                const int my_page = __shfl_sync(0xffffffffu, page, pg);
-                const bool mine = (good >> pg) & 1u;
-                const uint32_t tile_bytes = (uint32_t)__popc(good) * Cfg::kHalves * kPieceBytes;
-                const char* src = p.pool + ((int64_t)my_page * p.Hkv + it.kv_head) * (int64_t)(2 * Cfg::kHalves * kPieceBytes);
+            while (next_item()) {
+                __syncthreads();
+                const int32_t* bt = p.block_table + (int64_t)it.req * p.max_pages + it.key_begin / kPage;
+                bool ok = true;
+                for (int j = 0; j < n_tiles && ok; ++j) {
+                    const uint32_t tc = tile_ctr + j;
+                    const uint32_t s = tc & 1, par = (tc >> 1) & 1;
+                    const int n_keys = min(kTileKeys, it.key_end - (it.key_begin + j * kTileKeys));
+                    const int n_pages = (n_keys + kPage - 1) / kPage;
+                    const int page = (lane < n_pages) ? __ldg(bt + j * 8 + lane) : 0;
+                    const bool in_range = (uint32_t)page < (uint64_t)p.num_pages;
+                    const uint32_t good = __ballot_sync(0xffffffffu, lane < n_pages && in_range);
+                    if (__popc(good) != n_pages && lane == 0) atomicOr(&p.hdr->status, kStatusBounds);
+                    const int my_page = __shfl_sync(0xffffffffu, page, pg);
+                    const bool mine = (good >> pg) & 1u;
+                    const uint32_t tile_bytes = (uint32_t)__popc(good) * Cfg::kHalves * kPieceBytes;
+                    const char* src = p.pool + ((int64_t)my_page * p.Hkv + it.kv_head) * (int64_t)(2 * Cfg::kHalves * kPieceBytes);
 
-                ok = wait_all(bars + Bars::k_empty + 8 * s, par ^ 1, s_abort);
-                if (!ok) break;
-                if (lane == 0) mbar_expect_tx(bars + Bars::k_full + 8 * s, tile_bytes);
-                __syncwarp();
-                if (mine && which < Cfg::kHalves)
-                    bulk_g2s(sbase + Cfg::kOffK + s * Cfg::kKBytes + which * Cfg::kHalfBytes + pg * kPieceBytes,
-                             src + which * kPieceBytes, kPieceBytes, bars + Bars::k_full + 8 * s);
-
-                ok = wait_all(bars + Bars::v_empty + 8 * s, par ^ 1, s_abort);
-                if (!ok) break;
-                if (lane == 0) mbar_expect_tx(bars + Bars::v_full + 8 * s, tile_bytes);
-                __syncwarp();
-                if (mine && which >= 2 && which - 2 < Cfg::kHalves)
-                    bulk_g2s(sbase + Cfg::kOffV + s * Cfg::kVBytes + (which - 2) * Cfg::kHalfBytes + pg * kPieceBytes,
-                             src + (Cfg::kHalves + which - 2) * kPieceBytes, kPieceBytes, bars + Bars::v_full + 8 * s);
-            }
-        } else {
-            // =========================== MMA issue ===========================
-            bool ok = true;
-            const int n_x = has_b ? 2 : 1;
-            // S_x(j) = Q_x K(j)^T; the last tile to read K stage s releases it
-            auto issue_qk = [&](int j, int x) {
-                const uint32_t tc = tile_ctr + j;
-                const uint32_t s = tc & 1;
-                if (x == 0) {
-                    ok = wait_all(bars + Bars::k_full + 8 * s, (tc >> 1) & 1, s_abort);
-                    if (!ok) return;
-                    tc_fence_after();
-                }
-                if (lane == 0) {
-                    const uint32_t d_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
-#pragma unroll
-                    for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = (kk >> 2) * Cfg::kHalfBytes + (kk & 3) * 32;
-                        tc_mma_ss(d_addr, smem_desc(sbase + Cfg::kOffQ + x * Cfg::kQBytes + off, 16, 1024),
-                                  smem_desc(sbase + Cfg::kOffK + s * Cfg::kKBytes + off, 16, 1024), kIdescQK, kk > 0);
-                    }
-                    tc_commit(bars + Bars::s_full + 8 * x);
-                    if (x == n_x - 1) tc_commit(bars + Bars::k_empty + 8 * s);
-                }
-                __syncwarp();
-            };
-            for (int x = 0; x < n_x && ok; ++x) issue_qk(0, x);
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const uint32_t tc = tile_ctr + j;
-                const uint32_t s = tc & 1;
-                for (int x = 0; x < n_x && ok; ++x) {
-                    ok = wait_all(bars + Bars::p_ready + 8 * x, ((x ? tile_ctr_b : tile_ctr) + j) & 1, s_abort);
+                    ok = wait_all(bars + Bars::k_empty + 8 * s, par ^ 1, s_abort);
                     if (!ok) break;
+                    if (lane == 0) mbar_expect_tx(bars + Bars::k_full + 8 * s, tile_bytes);
+                    __syncwarp();
+                    if (mine && which < Cfg::kHalves)
+                        bulk_g2s(sbase + Cfg::kOffK + s * Cfg::kKBytes + which * Cfg::kHalfBytes + pg * kPieceBytes,
+                                 src + which * kPieceBytes, kPieceBytes, bars + Bars::k_full + 8 * s);
+
+                    ok = wait_all(bars + Bars::v_empty + 8 * s, par ^ 1, s_abort);
+                    if (!ok) break;
+                    if (lane == 0) mbar_expect_tx(bars + Bars::v_full + 8 * s, tile_bytes);
+                    __syncwarp();
+                    if (mine && which >= 2 && which - 2 < Cfg::kHalves)
+                        bulk_g2s(sbase + Cfg::kOffV + s * Cfg::kVBytes + (which - 2) * Cfg::kHalfBytes + pg * kPieceBytes,
+                                 src + (Cfg::kHalves + which - 2) * kPieceBytes, kPieceBytes, bars + Bars::v_full + 8 * s);
+                }
+                advance();
+            }
+        } else if (warp == kMmaWarp) {
+            // ================================================================
+            // MMA issue
+            // ================================================================
+            // descriptors without their start address; a k-step adds its byte offset / 16 to the low word
+            const uint64_t desc_kmajor = smem_desc(0, 16, 1024);
+            const uint64_t desc_v = smem_desc(0, Cfg::kHalfBytes, 1024);
+            while (next_item()) {
+                __syncthreads();
+                bool ok = true;
+                const int n_x = has_b ? 2 : 1;
+                // S_x(j) = Q_x K(j)^T; the last tile to read K stage s releases it
+                auto issue_qk = [&](int j, int x) {
+                    const uint32_t tc = tile_ctr + j;
+                    const uint32_t s = tc & 1;
                     if (x == 0) {
-                        ok = wait_all(bars + Bars::v_full + 8 * s, (tc >> 1) & 1, s_abort);
-                        if (!ok) break;
+                        ok = wait_all(bars + Bars::k_full + 8 * s, (tc >> 1) & 1, s_abort);
+                        if (!ok) return;
+                        tc_fence_after();
                     }
-                    tc_fence_after();
                     if (lane == 0) {
-                        // O_x += P_x V(j): P_x sits in S_x's first 64 columns, two bf16 per column
-                        const uint32_t a_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
-                        const uint32_t d_addr = tmem + Cfg::kColO + x * Cfg::kColTile;
+                        const uint32_t d_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
+                        const uint64_t qd = desc_kmajor + ((sbase + Cfg::kOffQ + x * Cfg::kQBytes) >> 4);
+                        const uint64_t kd = desc_kmajor + ((sbase + Cfg::kOffK + s * Cfg::kKBytes) >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < kTileKeys / 16; ++kk) {
-                            const uint64_t bdesc = smem_desc(sbase + Cfg::kOffV + s * Cfg::kVBytes + kk * 2048, Cfg::kHalfBytes, 1024);
-                            tc_mma_ts(d_addr, a_addr + kk * 8, bdesc, kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint32_t off = ((kk >> 2) * Cfg::kHalfBytes + (kk & 3) * 32) >> 4;
+                            tc_mma_ss(d_addr, qd + off, kd + off, kIdescQK, kk > 0);
                         }
-                        if (j == n_tiles - 1) tc_commit(bars + Bars::o_done + 8 * x);
-                        if (x == n_x - 1) tc_commit(bars + Bars::v_empty + 8 * s);
+                        tc_commit(bars + Bars::s_full + 8 * x);
+                        if (x == n_x - 1) tc_commit(bars + Bars::k_empty + 8 * s);
                     }
                     __syncwarp();
-                    // the tensor pipe runs this thread's MMAs in issue order, so S_x may be
-                    // overwritten by the next QK^T right behind the PV that reads P_x
-                    if (j + 1 < n_tiles) issue_qk(j + 1, x);
+                };
+                for (int x = 0; x < n_x && ok; ++x) issue_qk(0, x);
+                for (int j = 0; j < n_tiles && ok; ++j) {
+                    const uint32_t tc = tile_ctr + j;
+                    const uint32_t s = tc & 1;
+                    for (int x = 0; x < n_x && ok; ++x) {
+                        ok = wait_all(bars + Bars::p_ready + 8 * x, ((x ? tile_ctr_b : tile_ctr) + j) & 1, s_abort);
+                        if (!ok) break;
+                        if (x == 0) {
+                            ok = wait_all(bars + Bars::v_full + 8 * s, (tc >> 1) & 1, s_abort);
+                            if (!ok) break;
+                        }
+                        tc_fence_after();
+                        if (lane == 0) {
+                            // O_x += P_x V(j): P_x sits in S_x's first 64 columns, two bf16 per column
+                            const uint32_t a_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
+                            const uint32_t d_addr = tmem + Cfg::kColO + x * Cfg::kColTile;
+                            const uint64_t vd = desc_v + ((sbase + Cfg::kOffV + s * Cfg::kVBytes) >> 4);
+#pragma unroll
+                            for (int kk = 0; kk < kTileKeys / 16; ++kk)
+                                tc_mma_ts(d_addr, a_addr + kk * 8, vd + kk * (2048 >> 4), kIdescPV, (j > 0 || kk > 0) ? 1u : 0u);
+                            if (j == n_tiles - 1) tc_commit(bars + Bars::o_done + 8 * x);
+                            if (x == n_x - 1) tc_commit(bars + Bars::v_empty + 8 * s);
+                        }
+                        __syncwarp();
+                        // the tensor pipe runs this thread's MMAs in issue order, so S_x may be
+                        // overwritten by the next QK^T right behind the PV that reads P_x
+                        if (j + 1 < n_tiles) issue_qk(j + 1, x);
+                    }
                 }
+                advance();
             }
-        }
-        tile_ctr += n_tiles;
-        ++item_ctr;
-        if (has_b) {
-            tile_ctr_b += n_tiles;
-            ++item_ctr_b;
+        } else {
+            // the warpgroup's two spare warps only keep the CTA-wide barriers complete
+            while (next_item()) {
+                __syncthreads();
+                advance();
+            }
         }
     }
 
