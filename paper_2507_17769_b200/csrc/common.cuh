@@ -132,6 +132,8 @@ struct DeviceWork {       // pointers into the workspace for one run
     float* part_lse;
     float* part_o;
     int32_t n_units, n_prefill, n_merge;
+    const int32_t* prefill_cta_start;  // static prefill partition (n_prefill_ctas + 1 entries), unused when 0
+    int32_t n_prefill_ctas;
 };
 
 struct RunArgs {

@@ -17,7 +17,7 @@ __global__ void __launch_bounds__(128) merge_kernel(const MergeEntry* __restrict
     const MergeEntry e = entries[blockIdx.x];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int rows = e.n_tok * G;
-    for (int rw = warp; rw < rows; rw += 4) {
+    for (int rw = warp + 4 * blockIdx.y; rw < rows; rw += 4 * gridDim.y) {
         const int i = rw / G, hh = rw % G;
         const int64_t slot0 = (int64_t)e.base + (int64_t)i * G + hh;
         float M = -INFINITY;
@@ -53,10 +53,12 @@ __global__ void __launch_bounds__(128) merge_kernel(const MergeEntry* __restrict
 ps_status launch_merge(const RunArgs& a) {
     if (a.w.n_merge == 0) return PS_OK;
     const int Hq = a.shape.n_q_heads, G = Hq / a.shape.n_kv_heads;
+    // blockIdx.x = merge entry; blockIdx.y spreads an entry's rows (up to 256 for a prefill item) over blocks
+    const dim3 grid(a.w.n_merge, a.w.n_prefill > 0 ? 16 : 1);
     if (a.shape.head_dim == 128)
-        merge_kernel<128><<<a.w.n_merge, 128, 0, a.stream>>>(a.w.merge, a.w.part_lse, a.w.part_o, a.out, a.lse, Hq, G);
+        merge_kernel<128><<<grid, 128, 0, a.stream>>>(a.w.merge, a.w.part_lse, a.w.part_o, a.out, a.lse, Hq, G);
     else
-        merge_kernel<64><<<a.w.n_merge, 128, 0, a.stream>>>(a.w.merge, a.w.part_lse, a.w.part_o, a.out, a.lse, Hq, G);
+        merge_kernel<64><<<grid, 128, 0, a.stream>>>(a.w.merge, a.w.part_lse, a.w.part_o, a.out, a.lse, Hq, G);
     PS_CUDA_TRY(cudaGetLastError());
     return PS_OK;
 }

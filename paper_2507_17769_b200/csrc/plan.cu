@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <chrono>
 #include <cstdlib>
+#include <cmath>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -31,10 +32,11 @@ struct ps_plan {
     std::vector<DecodeUnit> units;
     std::vector<PrefillItem> prefill;
     std::vector<MergeEntry> merge;
+    std::vector<int32_t> prefill_cta_start;  // static partition: CTA b runs items [start[b], start[b+1]); empty = dynamic queue
     std::vector<int32_t> prior;  // kept for item inspection
     ps_plan_info info{};
     // workspace layout
-    size_t off_pieces = 0, off_units = 0, off_prefill = 0, off_merge = 0, image_bytes = 0;
+    size_t off_pieces = 0, off_units = 0, off_prefill = 0, off_merge = 0, off_cta_start = 0, image_bytes = 0;
     size_t off_part_lse = 0, off_part_o = 0, ws_bytes = 0;
     // pinned staging image of [0, image_bytes)
     char* pinned = nullptr;
@@ -116,6 +118,11 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
     }
 }
 
+// Cost model of the prefill kernel in units of one 128-key tile step: an item pays a fixed
+// overhead (Q load, pipeline fill, epilogue) plus one unit per key tile.
+constexpr double kPrefillFixedCost = 2.0;
+constexpr double kPrefillMinCtaCost = 8.0;  // do not spread the work thinner than this per CTA
+
 static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len, const std::vector<int32_t>& q_start,
                          const ps_plan_opts* opts, int64_t* n_slots) {
     const int Hkv = pl->shape.n_kv_heads, G = pl->shape.n_q_heads / Hkv;
@@ -125,32 +132,76 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
     int64_t total_key_tiles = 0;
     for (int r = 0; r < pl->n; ++r) {
         if (q_len[r] <= 1) continue;
-        for (int t0 = 0; t0 < q_len[r]; t0 += tile_tok) {
-            const int n_tok = std::min(tile_tok, q_len[r] - t0);
-            const int first_pos = prior[r] + t0;
-            const int kt = (first_pos + n_tok + kPrefillKeyTile - 1) / kPrefillKeyTile;
-            for (int g = 0; g < Hkv; ++g) {
+        for (int g = 0; g < Hkv; ++g)
+            for (int t0 = 0; t0 < q_len[r]; t0 += tile_tok) {
+                const int n_tok = std::min(tile_tok, q_len[r] - t0);
+                const int first_pos = prior[r] + t0;
+                const int kt = (first_pos + n_tok + kPrefillKeyTile - 1) / kPrefillKeyTile;
                 tiles.push_back(Tile{r, g, t0, n_tok, first_pos, kt});
                 total_key_tiles += kt;
             }
-        }
     }
+    pl->prefill_cta_start.clear();
     if (tiles.empty()) return;
-    int seg_tiles;  // key tiles per item
-    if (opts && opts->prefill_segment_tokens > 0) {
-        seg_tiles = std::max(1, opts->prefill_segment_tokens / kPrefillKeyTile);
-    } else if ((int64_t)tiles.size() >= 2LL * pl->num_sms) {
-        seg_tiles = 1 << 30;
-    } else {
-        const int64_t target = 2LL * pl->num_sms;
-        seg_tiles = (int)std::max<int64_t>(4, (total_key_tiles + target - 1) / target);
-    }
-    pl->info.prefill_segment_tokens = seg_tiles >= (1 << 22) ? 0 : seg_tiles * kPrefillKeyTile;
 
-    for (const Tile& t : tiles) {
-        const int n_seg = (t.key_tiles + seg_tiles - 1) / seg_tiles;
-        // spread the key tiles evenly over the segments
-        const int base_tiles = t.key_tiles / n_seg, extra = t.key_tiles % n_seg;
+    // cut[i] = key-tile indices at which tile i is cut into pieces (ascending, exclusive of 0 and key_tiles)
+    std::vector<std::vector<int>> cuts(tiles.size());
+    // owner CTA of the first piece of each tile and of each following piece, for the static partition
+    bool static_partition = false;
+    if (opts && opts->prefill_segment_tokens > 0) {
+        const int seg_tiles = std::max(1, opts->prefill_segment_tokens / kPrefillKeyTile);
+        pl->info.prefill_segment_tokens = seg_tiles * kPrefillKeyTile;
+        for (size_t i = 0; i < tiles.size(); ++i) {
+            const int n_seg = (tiles[i].key_tiles + seg_tiles - 1) / seg_tiles;
+            const int base_tiles = tiles[i].key_tiles / n_seg, extra = tiles[i].key_tiles % n_seg;
+            int kt0 = 0;
+            for (int s = 0; s + 1 < n_seg; ++s) {
+                kt0 += base_tiles + (s < extra ? 1 : 0);
+                cuts[i].push_back(kt0);
+            }
+        }
+    } else if ((int64_t)tiles.size() < 4LL * pl->num_sms) {
+        // Few items per SM: give every CTA an equal share of the flattened (item, key tile) cost
+        // line, cutting items where a share ends.  Only the cut items need the merge.
+        static_partition = true;
+        double total = 0;
+        for (const Tile& t : tiles) total += kPrefillFixedCost + t.key_tiles;
+        const int n_cta = (int)std::max<double>(1, std::min<double>(pl->num_sms, total / kPrefillMinCtaCost));
+        const double quota = total / n_cta;
+        pl->prefill_cta_start.assign(1, 0);
+        double cum = 0, boundary = quota;
+        int n_items = 0, cta = 0;
+        for (size_t i = 0; i < tiles.size(); ++i) {
+            const int kt = tiles[i].key_tiles;
+            const double tile_end = cum + kPrefillFixedCost + kt;
+            int kt0 = 0;
+            while (cta < n_cta - 1 && boundary < tile_end - 0.5) {
+                int cut = (int)std::lround(boundary - cum - kPrefillFixedCost);
+                cut = std::max(cut, kt0);
+                if (cut >= kt) break;
+                if (cut > kt0) {
+                    cuts[i].push_back(cut);
+                    kt0 = cut;
+                    ++n_items;
+                }
+                ++cta;
+                pl->prefill_cta_start.push_back(n_items);
+                boundary += quota;
+            }
+            ++n_items;
+            cum = tile_end;
+            while (cta < n_cta - 1 && boundary <= cum + 0.5) {
+                ++cta;
+                pl->prefill_cta_start.push_back(n_items);
+                boundary += quota;
+            }
+        }
+        pl->prefill_cta_start.push_back(n_items);
+    }
+
+    for (size_t i = 0; i < tiles.size(); ++i) {
+        const Tile& t = tiles[i];
+        const int n_seg = (int)cuts[i].size() + 1;
         const int visible = t.first_pos + t.n_tok;
         int32_t slot_base = -1;
         if (n_seg > 1) {
@@ -165,26 +216,27 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
             pl->merge.push_back(me);
             *n_slots += (int64_t)n_seg * t.n_tok * G;
         }
-        int kt0 = 0;
         for (int s = 0; s < n_seg; ++s) {
-            const int nt = base_tiles + (s < extra ? 1 : 0);
+            const int kt0 = s == 0 ? 0 : cuts[i][s - 1];
+            const int kt1 = s == n_seg - 1 ? t.key_tiles : cuts[i][s];
             PrefillItem it{};
             it.req = t.r;
             it.kv_head = t.g;
             it.key_begin = kt0 * kPrefillKeyTile;
-            it.key_end = std::min(visible, (kt0 + nt) * kPrefillKeyTile);
+            it.key_end = std::min(visible, kt1 * kPrefillKeyTile);
             it.q_tok = q_start[t.r] + t.tok0;
             it.n_tok = t.n_tok;
             it.part_slot = n_seg > 1 ? slot_base + s * t.n_tok * G : -1;
             it.first_pos = t.first_pos;
             pl->prefill.push_back(it);
-            kt0 += nt;
         }
     }
-    // longest first: the dynamic queue then finishes with the short items
-    std::stable_sort(pl->prefill.begin(), pl->prefill.end(), [](const PrefillItem& a, const PrefillItem& b) {
-        return (a.key_end - a.key_begin) > (b.key_end - b.key_begin);
-    });
+    if (!static_partition) {
+        // dynamic queue: longest first, so that it finishes with the short items
+        std::stable_sort(pl->prefill.begin(), pl->prefill.end(), [](const PrefillItem& a, const PrefillItem& b) {
+            return (a.key_end - a.key_begin) > (b.key_end - b.key_begin);
+        });
+    }
 }
 
 extern "C" {
@@ -258,6 +310,7 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     pl->off_units = off;    off = align_up(off + pl->units.size() * sizeof(DecodeUnit), 256);
     pl->off_prefill = off;  off = align_up(off + pl->prefill.size() * sizeof(PrefillItem), 256);
     pl->off_merge = off;    off = align_up(off + pl->merge.size() * sizeof(MergeEntry), 256);
+    pl->off_cta_start = off; off = align_up(off + pl->prefill_cta_start.size() * sizeof(int32_t), 256);
     pl->image_bytes = off;
     pl->off_part_lse = off; off = align_up(off + (size_t)n_slots * sizeof(float), 256);
     pl->off_part_o = off;   off = align_up(off + (size_t)n_slots * d * sizeof(float), 256);
@@ -292,6 +345,8 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     if (!pl->units.empty()) memcpy(pl->pinned + pl->off_units, pl->units.data(), pl->units.size() * sizeof(DecodeUnit));
     if (!pl->prefill.empty()) memcpy(pl->pinned + pl->off_prefill, pl->prefill.data(), pl->prefill.size() * sizeof(PrefillItem));
     if (!pl->merge.empty()) memcpy(pl->pinned + pl->off_merge, pl->merge.data(), pl->merge.size() * sizeof(MergeEntry));
+    if (!pl->prefill_cta_start.empty())
+        memcpy(pl->pinned + pl->off_cta_start, pl->prefill_cta_start.data(), pl->prefill_cta_start.size() * sizeof(int32_t));
 
     pl->info.n_decode_items = (int32_t)pl->pieces.size();
     pl->info.n_prefill_items = (int32_t)pl->prefill.size();
@@ -389,6 +444,8 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     a.w.n_units = (int32_t)pl->units.size();
     a.w.n_prefill = (int32_t)pl->prefill.size();
     a.w.n_merge = (int32_t)pl->merge.size();
+    a.w.prefill_cta_start = (const int32_t*)(ws + pl->off_cta_start);
+    a.w.n_prefill_ctas = pl->prefill_cta_start.empty() ? 0 : (int32_t)pl->prefill_cta_start.size() - 1;
 
     const bool rec = pl->timing && (size_t)(pl->timed_runs + 1) * 4 <= pl->tev.size();
     cudaEvent_t* ev = rec ? &pl->tev[(size_t)pl->timed_runs * 4] : nullptr;

@@ -167,6 +167,7 @@ struct PrefillParams {
     WsHeader* hdr;
     const PrefillItem* items;
     int32_t n_items;
+    const int32_t* cta_start;  // static partition: this CTA runs items [cta_start[b], cta_start[b + 1]); null = dynamic queue
     float* part_lse;
     float* part_o;
     int32_t Hq, Hkv, G;
@@ -239,8 +240,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
     PrefillItem it;
     int n_tiles = 0;
     bool has_b = false;
+    int static_cur = p.cta_start ? p.cta_start[blockIdx.x] : 0;
+    const int static_end = p.cta_start ? p.cta_start[blockIdx.x + 1] : 0;
     auto next_item = [&]() -> bool {
-        if (threadIdx.x == 0) *s_item = atomicAdd(&p.hdr->prefill_next, 1);
+        if (threadIdx.x == 0)
+            *s_item = p.cta_start ? (static_cur < static_end ? static_cur : p.n_items) : atomicAdd(&p.hdr->prefill_next, 1);
+        ++static_cur;
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
@@ -631,13 +636,14 @@ static ps_status launch_prefill_d(const RunArgs& a) {
     p.hdr = a.w.hdr;
     p.items = a.w.prefill;
     p.n_items = a.w.n_prefill;
+    p.cta_start = a.w.n_prefill_ctas > 0 ? a.w.prefill_cta_start : nullptr;
     p.part_lse = a.w.part_lse;
     p.part_o = a.w.part_o;
     p.Hq = a.shape.n_q_heads;
     p.Hkv = a.shape.n_kv_heads;
     p.G = p.Hq / p.Hkv;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
-    const int grid = a.w.n_prefill < a.num_sms ? a.w.n_prefill : a.num_sms;
+    const int grid = a.w.n_prefill_ctas > 0 ? a.w.n_prefill_ctas : (a.w.n_prefill < a.num_sms ? a.w.n_prefill : a.num_sms);
     prefill_kernel<D><<<grid, kThreads, Cfg::kSmemBytes, a.stream>>>(p);
     PS_CUDA_TRY(cudaGetLastError());
     return PS_OK;
