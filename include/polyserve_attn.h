@@ -182,8 +182,11 @@ ps_status ps_plan_get_items(const ps_plan *plan, int32_t *decode_items_out, int6
  * entries past a sequence's last page are never read.  workspace_dev: device
  * memory (256-byte aligned) of at least the plan's workspace bytes; its
  * contents need no initialisation and are scratch.  Asynchronous on `stream`:
- * one small host-to-device copy of the work list, then the decode, prefill
- * and merge kernels.  Two runs of the same plan must not overlap on the device.
+ * the work list is uploaded (on a stream of the plan's own, ordered against
+ * `stream` with events, into one of two slots of the workspace so that it can
+ * run under the previous run's kernels), then the prefill, decode and merge
+ * kernels run on `stream`.  Consecutive runs of one plan must be issued to the
+ * same stream, or be ordered by the caller: they share the partial buffers.
  * Returns host-detectable errors only (PS_ERR_INVALID, PS_ERR_WORKSPACE,
  * PS_ERR_CUDA); errors seen on the device are read with ps_plan_status.
  */

@@ -90,7 +90,14 @@ struct DecodePiece {
     int32_t q_tok;        // packed q token index
     int32_t part_slot;    // first partial slot (head 0 of the group), or -1: write final output
     int32_t kv_len;       // keys visible to the row
-    int32_t pad;
+    int32_t merge_idx;    // index into the decode merge records when part_slot >= 0
+};
+
+// A (request, kv head) whose keys were cut into n_seg pieces: partial (s, hh) is slot base + s * G + hh.
+// The decode warp that delivers the last piece combines them (arrival counted in a zeroed int per record).
+struct DecodeMerge {
+    int32_t base;
+    int32_t n_seg;
 };
 
 // A decode work unit: pieces [piece_begin, piece_end) processed by one warp.
@@ -129,6 +136,8 @@ struct DeviceWork {       // pointers into the workspace for one run
     const DecodeUnit* units;
     const PrefillItem* prefill;
     const MergeEntry* merge;
+    const DecodeMerge* dmerge;
+    int32_t* dmerge_cnt;
     float* part_lse;
     float* part_o;
     int32_t n_units, n_prefill, n_merge;

@@ -26,13 +26,15 @@ namespace {
 
 constexpr int kWarps = 8;
 constexpr int kRing = 8;  // unit ids in flight between the producer and consumer cursors of a warp
+constexpr int kDeferred = 8;  // merges a warp can postpone until its KV stream has drained
 
 template <int D>
 struct DecodeCfg {
     static constexpr int kBlockBytes = kPage * D * 2;      // K (or V) of one page, one kv head
     static constexpr int kStageBytes = 2 * kBlockBytes;    // K then V
     static constexpr int kStages = (D == 128) ? 3 : 6;
-    static constexpr int kSmemBytes = kWarps * kStages * kStageBytes + kWarps * kStages * 8 + kWarps * kRing * 4 + 1024;
+    static constexpr int kSmemBytes =
+        kWarps * kStages * kStageBytes + kWarps * kStages * 8 + kWarps * kRing * 4 + kWarps * kDeferred * 12 + 1024;
 };
 
 struct DecodeParams {
@@ -47,6 +49,8 @@ struct DecodeParams {
     const DecodePiece* pieces;
     const DecodeUnit* units;
     int32_t n_units;
+    const DecodeMerge* dmerge;
+    int32_t* dmerge_cnt;
     float* part_lse;
     float* part_o;
     int32_t Hq, Hkv, G;
@@ -66,6 +70,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kWarps * STAGES * Cfg::kStageBytes) + warp * STAGES;
     int32_t* ring = reinterpret_cast<int32_t*>(smem + (size_t)kWarps * STAGES * Cfg::kStageBytes + kWarps * STAGES * 8) +
                     warp * kRing;
+    int32_t* deferred = reinterpret_cast<int32_t*>(smem + (size_t)kWarps * STAGES * Cfg::kStageBytes + kWarps * STAGES * 8 +
+                                                   kWarps * kRing * 4) + warp * kDeferred * 3;
     const uint32_t stage0 = smem_u32(my_stages);
     const uint32_t bar0 = smem_u32(bars);
 
@@ -128,7 +134,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
 
     // ---- consumer cursor ----
     int C_piece = 0, C_piece_end = 0, C_page = 0, C_page_end = 0;
-    int C_qtok = 0, C_slot = -1, C_kvlen = 0, C_g = 0;
+    int C_qtok = 0, C_slot = -1, C_kvlen = 0, C_g = 0, C_midx = 0;
     bool have_piece = false, timed_out = false;
     uint32_t n_cons = 0, cseq = 0;
 
@@ -142,6 +148,42 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
     // ldmatrix row addresses (byte offsets inside a block, before the per-step unit term)
     const uint32_t k_tok_off = (uint32_t)(((mi & 1) * 8 + l7) * 128);
     const uint32_t v_tok_off = (uint32_t)(((mi >> 1) * 8 + l7) * 128);
+
+    // Combine the partials of merge record midx (output token qtok, kv head g), in segment order.
+    int n_deferred = 0;
+    auto combine = [&](int midx, int qtok, int g) {
+        __threadfence();
+        const DecodeMerge dm = p.dmerge[midx];
+        constexpr int V = D / 32;  // floats per lane
+        for (int hh = 0; hh < p.G; ++hh) {
+            float M = -INFINITY;
+            for (int s = 0; s < dm.n_seg; ++s) M = fmaxf(M, __ldcg(p.part_lse + dm.base + s * p.G + hh));
+            float acc[V];
+#pragma unroll
+            for (int v = 0; v < V; ++v) acc[v] = 0.f;
+            float denom = 0.f;
+            for (int s = 0; s < dm.n_seg; ++s) {
+                const int64_t slot = (int64_t)dm.base + s * p.G + hh;
+                const float w = __expf(__ldcg(p.part_lse + slot) - M);
+                denom += w;
+                const float* po = p.part_o + slot * D + lane * V;
+                if constexpr (V == 4) {
+                    const float4 x = __ldcg(reinterpret_cast<const float4*>(po));
+                    acc[0] += w * x.x; acc[1] += w * x.y; acc[2] += w * x.z; acc[3] += w * x.w;
+                } else {
+                    const float2 x = __ldcg(reinterpret_cast<const float2*>(po));
+                    acc[0] += w * x.x; acc[1] += w * x.y;
+                }
+            }
+            const float inv = 1.f / denom;
+            const int64_t orow = (int64_t)qtok * p.Hq + g * p.G + hh;
+            __nv_bfloat16* op = p.out + orow * D + lane * V;
+#pragma unroll
+            for (int v = 0; v < V; v += 2)
+                *reinterpret_cast<__nv_bfloat162*>(op + v) = __floats2bfloat162_rn(acc[v] * inv, acc[v + 1] * inv);
+            if (p.lse && lane == 0) p.lse[orow] = M + __logf(denom);
+        }
+    };
 
     auto finalize = [&]() {
         // column sums over the 8 row-groups of the fragment
@@ -193,6 +235,28 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
                 if (col < p.G) p.part_lse[C_slot + col] = lse0;
                 if (col + 1 < p.G) p.part_lse[C_slot + col + 1] = lse1;
             }
+            // The warp that delivers the last piece of a (request, kv head) combines all of its
+            // partials, always in segment order, so the result does not depend on which warp that is.
+            __threadfence();
+            __syncwarp();
+            int arrived = 0;
+            const DecodeMerge dm = p.dmerge[C_midx];
+            if (lane == 0) arrived = atomicAdd(&p.dmerge_cnt[C_midx], 1);
+            arrived = __shfl_sync(0xffffffffu, arrived, 0);
+            if (arrived == dm.n_seg - 1) {
+                // Combining now would stall this warp's KV stream on dependent L2 reads; queue it
+                // for after the stream has drained (done at once only if the queue is full).
+                if (n_deferred < kDeferred) {
+                    if (lane == 0) {
+                        deferred[3 * n_deferred + 0] = C_midx;
+                        deferred[3 * n_deferred + 1] = C_qtok;
+                        deferred[3 * n_deferred + 2] = C_g;
+                    }
+                    ++n_deferred;
+                } else {
+                    combine(C_midx, C_qtok, C_g);
+                }
+            }
         }
     };
 
@@ -217,6 +281,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
             C_qtok = b.x;
             C_slot = b.y;
             C_kvlen = b.z;
+            C_midx = b.w;
             have_piece = true;
             // Q^T as B fragments: thread holds head (lane / 4), d = 16 ks + 2 (lane % 4) + {0, 1} (+ 8)
             const int hh = lane >> 2;
@@ -309,6 +374,10 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
         produce();     // refill the stage just released
     }
 
+    if (!timed_out) {
+        __syncwarp();
+        for (int k = 0; k < n_deferred; ++k) combine(deferred[3 * k], deferred[3 * k + 1], deferred[3 * k + 2]);
+    }
     if (timed_out) {
         // let copies still in flight land before the CTA's shared memory is released
         for (uint32_t n = n_cons + 1; n < n_prod; ++n) mbar_wait(bar0 + 8 * (n % STAGES), (n / STAGES) & 1, 2000000u);
@@ -339,6 +408,8 @@ static ps_status launch_decode_d(const RunArgs& a) {
     p.pieces = a.w.pieces;
     p.units = a.w.units;
     p.n_units = a.w.n_units;
+    p.dmerge = a.w.dmerge;
+    p.dmerge_cnt = a.w.dmerge_cnt;
     p.part_lse = a.w.part_lse;
     p.part_o = a.w.part_o;
     p.Hq = a.shape.n_q_heads;

@@ -31,19 +31,30 @@ struct ps_plan {
     std::vector<DecodePiece> pieces;
     std::vector<DecodeUnit> units;
     std::vector<PrefillItem> prefill;
-    std::vector<MergeEntry> merge;
+    std::vector<MergeEntry> merge;       // combined by the merge kernel (prefill items cut into segments)
+    std::vector<DecodeMerge> dmerge;     // combined inside the decode kernel
+    int64_t decode_merge_rows = 0;
     std::vector<int32_t> prefill_cta_start;  // static partition: CTA b runs items [start[b], start[b+1]); empty = dynamic queue
     std::vector<int32_t> prior;  // kept for item inspection
     ps_plan_info info{};
     // workspace layout
-    size_t off_pieces = 0, off_units = 0, off_prefill = 0, off_merge = 0, off_cta_start = 0, image_bytes = 0;
+    size_t off_pieces = 0, off_units = 0, off_prefill = 0, off_merge = 0, off_cta_start = 0, off_dmerge = 0, off_dmerge_cnt = 0, image_bytes = 0;
     size_t off_part_lse = 0, off_part_o = 0, ws_bytes = 0;
     // pinned staging image of [0, image_bytes)
     char* pinned = nullptr;
     bool pinned_is_cuda = false;
     size_t pinned_cap = 0;
-    cudaEvent_t copied = nullptr;
+    // The work-list image is uploaded on a private stream into one of two slots at the head of the
+    // workspace, so that the upload for run i+1 overlaps the kernels of run i.
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_copied[2] = {nullptr, nullptr};  // slot's upload finished (copy stream)
+    cudaEvent_t ev_done[2] = {nullptr, nullptr};    // the run that used the slot finished (caller's stream)
+    cudaEvent_t ev_fence = nullptr;                  // caller's stream position, when the workspace changed
+    bool done_valid[2] = {false, false};
     bool copy_pending = false;
+    int last_slot = 0;
+    unsigned run_no = 0;
+    void* last_ws = nullptr;
     WsHeader* last_hdr = nullptr;
     // optional per-kernel timing: 4 events per recorded run (before prefill, after prefill, after decode, after merge)
     bool timing = false;
@@ -103,15 +114,15 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
             }
             const size_t cnt = pl->pieces.size() - first_piece;
             if (cnt > 1) {
-                MergeEntry me{};
-                me.q_tok = q_start[r];
-                me.n_tok = 1;
-                me.kv_head = g;
-                me.base = (int32_t)*n_slots;
-                me.n_seg = (int32_t)cnt;
-                me.seg_stride = G;
-                pl->merge.push_back(me);
-                for (size_t s = 0; s < cnt; ++s) pl->pieces[first_piece + s].part_slot = (int32_t)(*n_slots + (int64_t)s * G);
+                DecodeMerge dm{};
+                dm.base = (int32_t)*n_slots;
+                dm.n_seg = (int32_t)cnt;
+                for (size_t s = 0; s < cnt; ++s) {
+                    pl->pieces[first_piece + s].part_slot = (int32_t)(*n_slots + (int64_t)s * G);
+                    pl->pieces[first_piece + s].merge_idx = (int32_t)pl->dmerge.size();
+                }
+                pl->dmerge.push_back(dm);
+                pl->decode_merge_rows += G;
                 *n_slots += (int64_t)cnt * G;
             }
         }
@@ -272,8 +283,8 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     if (fresh) {
         pl = new (std::nothrow) ps_plan();
         if (!pl) return fail(PS_ERR_OOM, "host allocation failed");
-    } else if (pl->copy_pending && pl->copied) {
-        cudaError_t e = cudaEventSynchronize(pl->copied);
+    } else if (pl->copy_pending && pl->ev_copied[pl->last_slot]) {
+        cudaError_t e = cudaEventSynchronize(pl->ev_copied[pl->last_slot]);
         if (e != cudaSuccess) return fail(PS_ERR_CUDA, "cudaEventSynchronize failed: %s", cudaGetErrorString(e));
         pl->copy_pending = false;
     }
@@ -294,6 +305,8 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     pl->units.clear();
     pl->prefill.clear();
     pl->merge.clear();
+    pl->dmerge.clear();
+    pl->decode_merge_rows = 0;
     pl->prior.assign(prior_host, prior_host + n);
     pl->info = ps_plan_info{};
     int64_t n_slots = 0;
@@ -310,8 +323,11 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     pl->off_units = off;    off = align_up(off + pl->units.size() * sizeof(DecodeUnit), 256);
     pl->off_prefill = off;  off = align_up(off + pl->prefill.size() * sizeof(PrefillItem), 256);
     pl->off_merge = off;    off = align_up(off + pl->merge.size() * sizeof(MergeEntry), 256);
+    pl->off_dmerge = off;   off = align_up(off + pl->dmerge.size() * sizeof(DecodeMerge), 256);
+    pl->off_dmerge_cnt = off; off = align_up(off + pl->dmerge.size() * sizeof(int32_t), 256);
     pl->off_cta_start = off; off = align_up(off + pl->prefill_cta_start.size() * sizeof(int32_t), 256);
     pl->image_bytes = off;
+    off = 2 * pl->image_bytes;  // two image slots
     pl->off_part_lse = off; off = align_up(off + (size_t)n_slots * sizeof(float), 256);
     pl->off_part_o = off;   off = align_up(off + (size_t)n_slots * d * sizeof(float), 256);
     pl->ws_bytes = off;
@@ -334,10 +350,16 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
         }
         pl->pinned_cap = cap;
     }
-    if (!pl->copied && pl->pinned_is_cuda) {
-        if (cudaEventCreateWithFlags(&pl->copied, cudaEventDisableTiming) != cudaSuccess) {
+    if (!pl->copy_stream && pl->pinned_is_cuda) {
+        bool ok = cudaStreamCreateWithFlags(&pl->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+        for (int b = 0; b < 2 && ok; ++b)
+            ok = cudaEventCreateWithFlags(&pl->ev_copied[b], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&pl->ev_done[b], cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaEventCreateWithFlags(&pl->ev_fence, cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
             (void)cudaGetLastError();
-            pl->copied = nullptr;
+            if (pl->copy_stream) cudaStreamDestroy(pl->copy_stream);
+            pl->copy_stream = nullptr;  // uploads then go on the caller's stream
         }
     }
     memset(pl->pinned, 0, 256);
@@ -345,12 +367,16 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     if (!pl->units.empty()) memcpy(pl->pinned + pl->off_units, pl->units.data(), pl->units.size() * sizeof(DecodeUnit));
     if (!pl->prefill.empty()) memcpy(pl->pinned + pl->off_prefill, pl->prefill.data(), pl->prefill.size() * sizeof(PrefillItem));
     if (!pl->merge.empty()) memcpy(pl->pinned + pl->off_merge, pl->merge.data(), pl->merge.size() * sizeof(MergeEntry));
+    if (!pl->dmerge.empty()) {
+        memcpy(pl->pinned + pl->off_dmerge, pl->dmerge.data(), pl->dmerge.size() * sizeof(DecodeMerge));
+        memset(pl->pinned + pl->off_dmerge_cnt, 0, pl->dmerge.size() * sizeof(int32_t));  // arrival counters start at zero
+    }
     if (!pl->prefill_cta_start.empty())
         memcpy(pl->pinned + pl->off_cta_start, pl->prefill_cta_start.data(), pl->prefill_cta_start.size() * sizeof(int32_t));
 
     pl->info.n_decode_items = (int32_t)pl->pieces.size();
     pl->info.n_prefill_items = (int32_t)pl->prefill.size();
-    int64_t merge_rows = 0;
+    int64_t merge_rows = pl->decode_merge_rows;
     for (const MergeEntry& me : pl->merge) merge_rows += (int64_t)me.n_tok * (shape->n_q_heads / shape->n_kv_heads);
     pl->info.n_merge_rows = (int32_t)merge_rows;
     pl->info.n_partial_slots = n_slots;
@@ -363,8 +389,15 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
 
 ps_status ps_plan_free(ps_plan* pl) {
     if (!pl) return PS_OK;
-    if (pl->copy_pending && pl->copied) cudaEventSynchronize(pl->copied);
-    if (pl->copied) cudaEventDestroy(pl->copied);
+    if (pl->copy_stream) {
+        cudaStreamSynchronize(pl->copy_stream);
+        cudaStreamDestroy(pl->copy_stream);
+    }
+    for (int b = 0; b < 2; ++b) {
+        if (pl->ev_copied[b]) cudaEventDestroy(pl->ev_copied[b]);
+        if (pl->ev_done[b]) cudaEventDestroy(pl->ev_done[b]);
+    }
+    if (pl->ev_fence) cudaEventDestroy(pl->ev_fence);
     for (cudaEvent_t e : pl->tev) cudaEventDestroy(e);
     if (pl->pinned) { if (pl->pinned_is_cuda) cudaFreeHost(pl->pinned); else free(pl->pinned); }
     delete pl;
@@ -413,12 +446,28 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     const KvPool& pool = pool_of(kv);
     if (memcmp(&pool.shape, &pl->shape, sizeof(ps_shape)) != 0) return fail(PS_ERR_INVALID, "plan and pool shapes differ");
     cudaStream_t s = (cudaStream_t)stream;
-    char* ws = (char*)workspace_dev;
-    PS_CUDA_TRY(cudaMemcpyAsync(ws, pl->pinned, pl->image_bytes, cudaMemcpyHostToDevice, s));
-    if (pl->copied) {
-        PS_CUDA_TRY(cudaEventRecord(pl->copied, s));
+    char* const ws_base = (char*)workspace_dev;
+    const int slot = (int)(pl->run_no++ & 1u);
+    char* ws = ws_base + (size_t)slot * pl->image_bytes;  // this run's image slot; partials are addressed from ws_base
+    if (pl->copy_stream) {
+        cudaStream_t cs = pl->copy_stream;
+        if (pl->last_ws == workspace_dev && pl->done_valid[slot]) {
+            // same workspace as before: the slot is free once the run two calls ago has finished
+            PS_CUDA_TRY(cudaStreamWaitEvent(cs, pl->ev_done[slot], 0));
+        } else {
+            // first use of this memory: order the upload after everything already on the caller's stream
+            PS_CUDA_TRY(cudaEventRecord(pl->ev_fence, s));
+            PS_CUDA_TRY(cudaStreamWaitEvent(cs, pl->ev_fence, 0));
+            if (pl->last_ws != workspace_dev) pl->done_valid[0] = pl->done_valid[1] = false;
+        }
+        PS_CUDA_TRY(cudaMemcpyAsync(ws, pl->pinned, pl->image_bytes, cudaMemcpyHostToDevice, cs));
+        PS_CUDA_TRY(cudaEventRecord(pl->ev_copied[slot], cs));
+        PS_CUDA_TRY(cudaStreamWaitEvent(s, pl->ev_copied[slot], 0));
         pl->copy_pending = true;
+        pl->last_slot = slot;
+        pl->last_ws = workspace_dev;
     } else {
+        PS_CUDA_TRY(cudaMemcpyAsync(ws, pl->pinned, pl->image_bytes, cudaMemcpyHostToDevice, s));
         PS_CUDA_TRY(cudaStreamSynchronize(s));  // no event to guard the staging image: finish the copy now
     }
     pl->last_hdr = (WsHeader*)ws;
@@ -439,11 +488,13 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     a.w.units = (const DecodeUnit*)(ws + pl->off_units);
     a.w.prefill = (const PrefillItem*)(ws + pl->off_prefill);
     a.w.merge = (const MergeEntry*)(ws + pl->off_merge);
-    a.w.part_lse = (float*)(ws + pl->off_part_lse);
-    a.w.part_o = (float*)(ws + pl->off_part_o);
+    a.w.part_lse = (float*)(ws_base + pl->off_part_lse);
+    a.w.part_o = (float*)(ws_base + pl->off_part_o);
     a.w.n_units = (int32_t)pl->units.size();
     a.w.n_prefill = (int32_t)pl->prefill.size();
     a.w.n_merge = (int32_t)pl->merge.size();
+    a.w.dmerge = (const DecodeMerge*)(ws + pl->off_dmerge);
+    a.w.dmerge_cnt = (int32_t*)(ws + pl->off_dmerge_cnt);
     a.w.prefill_cta_start = (const int32_t*)(ws + pl->off_cta_start);
     a.w.n_prefill_ctas = pl->prefill_cta_start.empty() ? 0 : (int32_t)pl->prefill_cta_start.size() - 1;
 
@@ -460,6 +511,10 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     if (rec) {
         cudaEventRecord(ev[3], s);
         ++pl->timed_runs;
+    }
+    if (pl->copy_stream && st == PS_OK) {
+        PS_CUDA_TRY(cudaEventRecord(pl->ev_done[slot], s));
+        pl->done_valid[slot] = true;
     }
     return st;
 }
