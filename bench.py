@@ -229,7 +229,7 @@ def run_ours(args):
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     with ClockSampler(local_rank) as clocks:
-        ps.ps_plan_set_timing(pa._plan, min(args.steps, 4096))
+        # pass 1: the K timed steps (two events around the whole region)
         ev0.record(stream)
         t_host = time.perf_counter()
         for _ in range(args.steps):
@@ -237,9 +237,15 @@ def run_ours(args):
         host_ms = (time.perf_counter() - t_host) * 1e3 / args.steps
         ev1.record(stream)
         barrier()
-    local_ms = ev0.elapsed_time(ev1) / args.steps
-    pre_ms, dec_ms, mrg_ms, n_timed = ps.ps_plan_get_timing(pa._plan, stream.cuda_stream)
-    ps.ps_plan_set_timing(pa._plan, 0)
+        local_ms = ev0.elapsed_time(ev1) / args.steps
+        # pass 2: the same steps again with events around every kernel launch, for the per-kernel
+        # durations of the roofline (kept out of pass 1: each extra event costs device time)
+        n_kernel_steps = min(args.steps, 1000)
+        ps.ps_plan_set_timing(pa._plan, n_kernel_steps)
+        for _ in range(n_kernel_steps):
+            step()
+        pre_ms, dec_ms, mrg_ms, n_timed = ps.ps_plan_get_timing(pa._plan, stream.cuda_stream)
+        ps.ps_plan_set_timing(pa._plan, 0)
     pa.check()
     dec_bytes, pf_flops = float(batch.decode_bytes()), float(batch.prefill_flops())
     ms, units = reduce_over_ranks(local_ms, dec_bytes, world, dev)

@@ -152,20 +152,31 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
     // Combine the partials of merge record midx (output token qtok, kv head g), in segment order.
     int n_deferred = 0;
     auto combine = [&](int midx, int qtok, int g) {
-        __threadfence();
+        __syncwarp();  // lane 0's acquiring increment is ordered before every lane's partial loads
         const DecodeMerge dm = p.dmerge[midx];
         constexpr int V = D / 32;  // floats per lane
+        // The n_seg * G log-sum-exps are contiguous (segment-major, head-minor).  Lane i reads entries
+        // i, i + 32, ...; since G divides 32 they all belong to head i % G, so the per-head max and
+        // sum are reductions over the lanes that are congruent mod G.
+        const int n = dm.n_seg * p.G;
+        const float* lse_in = p.part_lse + dm.base;
+        float mx = -INFINITY;
+        for (int i = lane; i < n; i += 32) mx = fmaxf(mx, __ldcg(lse_in + i));
+        for (int off = p.G; off < 32; off <<= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        float den = 0.f;
+        for (int i = lane; i < n; i += 32) den += __expf(__ldcg(lse_in + i) - mx);
+        for (int off = p.G; off < 32; off <<= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
         for (int hh = 0; hh < p.G; ++hh) {
-            float M = -INFINITY;
-            for (int s = 0; s < dm.n_seg; ++s) M = fmaxf(M, __ldcg(p.part_lse + dm.base + s * p.G + hh));
+            const float M = __shfl_sync(0xffffffffu, mx, hh);
+            const float inv = 1.f / __shfl_sync(0xffffffffu, den, hh);
             float acc[V];
 #pragma unroll
             for (int v = 0; v < V; ++v) acc[v] = 0.f;
-            float denom = 0.f;
+            // fixed segment order; the loads of up to four segments are in flight together
+#pragma unroll 4
             for (int s = 0; s < dm.n_seg; ++s) {
                 const int64_t slot = (int64_t)dm.base + s * p.G + hh;
                 const float w = __expf(__ldcg(p.part_lse + slot) - M);
-                denom += w;
                 const float* po = p.part_o + slot * D + lane * V;
                 if constexpr (V == 4) {
                     const float4 x = __ldcg(reinterpret_cast<const float4*>(po));
@@ -175,13 +186,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
                     acc[0] += w * x.x; acc[1] += w * x.y;
                 }
             }
-            const float inv = 1.f / denom;
             const int64_t orow = (int64_t)qtok * p.Hq + g * p.G + hh;
             __nv_bfloat16* op = p.out + orow * D + lane * V;
 #pragma unroll
             for (int v = 0; v < V; v += 2)
                 *reinterpret_cast<__nv_bfloat162*>(op + v) = __floats2bfloat162_rn(acc[v] * inv, acc[v + 1] * inv);
-            if (p.lse && lane == 0) p.lse[orow] = M + __logf(denom);
+            if (p.lse && lane == 0) p.lse[orow] = M + __logf(1.f / inv);
         }
     };
 
@@ -237,11 +247,14 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
             }
             // The warp that delivers the last piece of a (request, kv head) combines all of its
             // partials, always in segment order, so the result does not depend on which warp that is.
-            __threadfence();
+            // Release: the warp barrier orders every lane's partial stores before lane 0's
+            // acq_rel increment, which the combining warp's increment (acquire) observes.
             __syncwarp();
             int arrived = 0;
             const DecodeMerge dm = p.dmerge[C_midx];
-            if (lane == 0) arrived = atomicAdd(&p.dmerge_cnt[C_midx], 1);
+            if (lane == 0)
+                asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;"
+                             : "=r"(arrived) : "l"(p.dmerge_cnt + C_midx) : "memory");
             arrived = __shfl_sync(0xffffffffu, arrived, 0);
             if (arrived == dm.n_seg - 1) {
                 // Combining now would stall this warp's KV stream on dependent L2 reads; queue it
