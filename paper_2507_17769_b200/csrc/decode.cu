@@ -18,13 +18,23 @@
 //     spanning several (request, kv head) pieces) fetched from one atomic
 //     counter; the producer side of the warp runs STAGES pages ahead of the
 //     consumer side, across piece and unit boundaries.
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace ps {
 
 namespace {
 
-constexpr int kWarps = 8;
+#ifndef PS_DECODE_WARPS
+#define PS_DECODE_WARPS 12
+#endif
+#ifndef PS_DECODE_STAGES
+#define PS_DECODE_STAGES 2
+#endif
+// streaming warps per CTA (one CTA per SM) and ring depth per warp: 12 x 2 x 8 KB = 192 KB in flight per SM;
+// measured on B200: 12 x 2 and 10 x 2 beat 8 x 3, 6 x 4 and 4 x 6 by 2-6 %
+constexpr int kWarps = PS_DECODE_WARPS;
 constexpr int kRing = 8;  // unit ids in flight between the producer and consumer cursors of a warp
 constexpr int kDeferred = 8;  // merges a warp can postpone until its KV stream has drained
 
@@ -32,7 +42,7 @@ template <int D>
 struct DecodeCfg {
     static constexpr int kBlockBytes = kPage * D * 2;      // K (or V) of one page, one kv head
     static constexpr int kStageBytes = 2 * kBlockBytes;    // K then V
-    static constexpr int kStages = (D == 128) ? 3 : 6;
+    static constexpr int kStages = (D == 128) ? PS_DECODE_STAGES : 2 * PS_DECODE_STAGES;  // 8 KB (4 KB) stages per warp
     static constexpr int kSmemBytes =
         kWarps * kStages * kStageBytes + kWarps * kStages * 8 + kWarps * kRing * 4 + kWarps * kDeferred * 12 + 1024;
 };
@@ -166,33 +176,56 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
         float den = 0.f;
         for (int i = lane; i < n; i += 32) den += __expf(__ldcg(lse_in + i) - mx);
         for (int off = p.G; off < 32; off <<= 1) den += __shfl_xor_sync(0xffffffffu, den, off);
-        for (int hh = 0; hh < p.G; ++hh) {
-            const float M = __shfl_sync(0xffffffffu, mx, hh);
-            const float inv = 1.f / __shfl_sync(0xffffffffu, den, hh);
-            float acc[V];
+        // All heads at once: lane -> (head hh, slice of d); a lane owns D * G / 32 consecutive floats
+        // of its head's row, so every segment costs it a few independent 16-byte loads.
+        const int lanes_per_head = 32 / p.G;
+        const int hh = lane / lanes_per_head, part = lane % lanes_per_head;
+        const float M = __shfl_sync(0xffffffffu, mx, hh);
+        const float inv = 1.f / __shfl_sync(0xffffffffu, den, hh);
+        const int64_t orow = (int64_t)qtok * p.Hq + g * p.G + hh;
+        auto run = [&](auto nvec_tag) {
+            constexpr int NV = decltype(nvec_tag)::value;  // float4 per lane
+            float4 acc[NV];
 #pragma unroll
-            for (int v = 0; v < V; ++v) acc[v] = 0.f;
-            // fixed segment order; the loads of up to four segments are in flight together
-#pragma unroll 4
-            for (int s = 0; s < dm.n_seg; ++s) {
+            for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+            for (int s = 0; s < dm.n_seg; ++s) {  // fixed segment order
                 const int64_t slot = (int64_t)dm.base + s * p.G + hh;
                 const float w = __expf(__ldcg(p.part_lse + slot) - M);
-                const float* po = p.part_o + slot * D + lane * V;
-                if constexpr (V == 4) {
-                    const float4 x = __ldcg(reinterpret_cast<const float4*>(po));
-                    acc[0] += w * x.x; acc[1] += w * x.y; acc[2] += w * x.z; acc[3] += w * x.w;
-                } else {
-                    const float2 x = __ldcg(reinterpret_cast<const float2*>(po));
-                    acc[0] += w * x.x; acc[1] += w * x.y;
+                const float4* po = reinterpret_cast<const float4*>(p.part_o + slot * D) + part * NV;
+#pragma unroll
+                for (int v = 0; v < NV; ++v) {
+                    const float4 x = __ldcg(po + v);
+                    acc[v].x += w * x.x; acc[v].y += w * x.y; acc[v].z += w * x.z; acc[v].w += w * x.w;
                 }
             }
-            const int64_t orow = (int64_t)qtok * p.Hq + g * p.G + hh;
-            __nv_bfloat16* op = p.out + orow * D + lane * V;
+            uint2* op = reinterpret_cast<uint2*>(p.out + orow * D) + part * NV;
 #pragma unroll
-            for (int v = 0; v < V; v += 2)
-                *reinterpret_cast<__nv_bfloat162*>(op + v) = __floats2bfloat162_rn(acc[v] * inv, acc[v + 1] * inv);
-            if (p.lse && lane == 0) p.lse[orow] = M + __logf(1.f / inv);
+            for (int v = 0; v < NV; ++v)
+                op[v] = make_uint2(pack_bf16(acc[v].x * inv, acc[v].y * inv), pack_bf16(acc[v].z * inv, acc[v].w * inv));
+        };
+        // NV = D * G / 128: one float4 at (D, G) = (64, 2) or (128, 1) up to eight at (128, 8)
+        switch (D * p.G / 128) {
+            case 8: run(std::integral_constant<int, 8>{}); break;
+            case 4: run(std::integral_constant<int, 4>{}); break;
+            case 2: run(std::integral_constant<int, 2>{}); break;
+            case 1: run(std::integral_constant<int, 1>{}); break;
+            default: {  // D = 64, G = 1: half a float4 per lane -- let the first 16 lanes take one each
+                if (lane < 16) {
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int s = 0; s < dm.n_seg; ++s) {
+                        const int64_t slot = (int64_t)dm.base + s;
+                        const float w = __expf(__ldcg(p.part_lse + slot) - __shfl_sync(0xffffu, mx, 0));
+                        const float4 x = __ldcg(reinterpret_cast<const float4*>(p.part_o + slot * D) + lane);
+                        acc.x += w * x.x; acc.y += w * x.y; acc.z += w * x.z; acc.w += w * x.w;
+                    }
+                    const float inv1 = 1.f / __shfl_sync(0xffffu, den, 0);
+                    reinterpret_cast<uint2*>(p.out + ((int64_t)qtok * p.Hq + g) * D)[lane] =
+                        make_uint2(pack_bf16(acc.x * inv1, acc.y * inv1), pack_bf16(acc.z * inv1, acc.w * inv1));
+                }
+            }
         }
+        if (p.lse && part == 0 && hh < p.G) p.lse[orow] = M + __logf(1.f / inv);
     };
 
     auto finalize = [&]() {

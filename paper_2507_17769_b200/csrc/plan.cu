@@ -17,7 +17,7 @@ namespace ps {
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-constexpr int kDecodeUnitsPerWarp = 2;  // dynamic-queue units per resident warp
+constexpr int kDecodeUnitsPerWarp = 1;  // work units per resident warp (measured: 1 beats 2 and 3 on the decode-only batch)
 constexpr int kDecodeMinPages = 8;      // smallest decode unit (pages)
 constexpr int kPrefillKeyTile = 128;    // keys per tensor-core tile
 
