@@ -132,7 +132,7 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
 // Cost model of the prefill kernel in units of one 128-key tile step: an item pays a fixed
 // overhead (Q load, pipeline fill, epilogue) plus one unit per key tile.
 constexpr double kPrefillFixedCost = 2.0;
-constexpr double kPrefillMinCtaCost = 8.0;  // do not spread the work thinner than this per CTA
+constexpr double kPrefillMinCtaCost = 4.0;  // do not spread the work thinner than this per CTA (two key tiles)
 
 static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len, const std::vector<int32_t>& q_start,
                          const ps_plan_opts* opts, int64_t* n_slots) {

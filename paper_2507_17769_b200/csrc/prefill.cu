@@ -493,7 +493,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
             const int pg = lane >> 2, which = lane & 3;  // page in tile; 0/1 = K half 0/1, 2/3 = V half 0/1
             constexpr uint32_t kPieceBytes = kPage * 128;  // 16 tokens x 64 elements
             while (next_item()) {
-                __syncthreads();
+                // K and V do not depend on the Q tiles: the first tile's copies are issued before this
+                // warp joins the item's second CTA-wide barrier (Q tiles in shared memory)
+                bool joined = false;
                 const int32_t* bt = p.block_table + (int64_t)it.req * p.max_pages + it.key_begin / kPage;
                 bool ok = true;
                 for (int j = 0; j < n_tiles && ok; ++j) {
@@ -525,7 +527,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                     if (mine && which >= 2 && which - 2 < Cfg::kHalves)
                         bulk_g2s(sbase + Cfg::kOffV + s * Cfg::kVBytes + (which - 2) * Cfg::kHalfBytes + pg * kPieceBytes,
                                  src + (Cfg::kHalves + which - 2) * kPieceBytes, kPieceBytes, bars + Bars::v_full + 8 * s);
+                    if (!joined) {
+                        __syncthreads();
+                        joined = true;
+                    }
                 }
+                if (!joined) __syncthreads();
                 advance();
             }
         } else if (warp == kMmaWarp) {

@@ -215,7 +215,8 @@ extern "C" ps_status ps_profile_grid(const ps_shape* shape, const ps_grid_spec* 
                     make_draw(chunk, nd, m, seed, &dr);
                     const int n = (int)dr.prior.size();
                     const int64_t rot = std::min<int64_t>(
-                        kMaxRotate, std::max<int64_t>(1, std::min<int64_t>(cap_pages / dr.num_pages,
+                        std::min<int64_t>(kMaxRotate, std::max<int64_t>(1, cap_bt / (int64_t)dr.block_table.size())),
+                        std::max<int64_t>(1, std::min<int64_t>(cap_pages / dr.num_pages,
                                                                              (kRotateBytes + dr.num_pages * page_bytes - 1) / (dr.num_pages * page_bytes))));
                     bt_all.resize((size_t)rot * dr.block_table.size());
                     for (int64_t k = 0; k < rot; ++k)

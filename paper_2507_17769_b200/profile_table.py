@@ -1,0 +1,69 @@
+"""Emit the iteration-latency table the scheduler consults (paper section 4.5).
+
+    python -m paper_2507_17769_b200.profile_table [--out table.csv] [--seeds 27] [--iters 10] [--quick]
+
+Runs ps_profile_grid over chunk size x decode count x mean context (default:
+the 6 x 4 x 3 grid with 27 seeded length draws per cell) and prints, per cell,
+the median latency over the draws plus the table's two keys in the paper's
+terms: token batch size (chunk + decode rows) and KV-cache size (sum of
+kv_len).  Also reports how well latency at a fixed decode count is explained
+by an affine function of total KV tokens (the paper models decode attention
+time as a function of KV-cache size, section 3.4).
+"""
+from __future__ import annotations
+
+import argparse
+import statistics
+
+import numpy as np
+
+from . import binding as B
+
+CHUNKS = (64, 128, 256, 512, 1024, 2048)
+DECODES = (8, 32, 128, 256)
+CTXS = (512, 2048, 8192)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--out", default=None, help="CSV with one row per (cell, seed) draw")
+    ap.add_argument("--seeds", type=int, default=27)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--iters", type=int, default=10)
+    ap.add_argument("--quick", action="store_true", help="2 x 2 x 2 corner cells, 3 seeds")
+    ap.add_argument("--heads", default="32,8,128", help="n_q_heads,n_kv_heads,head_dim")
+    a = ap.parse_args()
+    hq, hkv, d = (int(x) for x in a.heads.split(","))
+    chunks, decodes, ctxs, seeds = CHUNKS, DECODES, CTXS, a.seeds
+    if a.quick:
+        chunks, decodes, ctxs, seeds = (64, 2048), (8, 256), (512, 8192), min(3, a.seeds)
+    rows = B.ps_profile_grid(B.make_shape(hq, hkv, d), chunks, decodes, ctxs, seeds, a.warmup, a.iters, 3000, a.out)
+    cells = {}
+    for r in rows:
+        cells.setdefault((r.chunk, r.n_decode, r.mean_ctx), []).append(r)
+    print("chunk n_dec mean_ctx | token_batch kv_tokens(med) | latency_us med [min..max over draws] | decode TB/s  prefill TFLOP/s (if each ran alone in that time)")
+    for (c, n, m), rs in cells.items():
+        lat = [r.latency_us for r in rs]
+        med = statistics.median(lat)
+        kv = statistics.median([r.kv_tokens for r in rs])
+        db = statistics.median([r.decode_bytes for r in rs])
+        pf = statistics.median([r.prefill_flops for r in rs])
+        print("%5d %5d %8d | %11d %14d | %9.1f [%8.1f .. %8.1f] | %6.2f %8.1f" %
+              (c, n, m, c + n, kv, med, min(lat), max(lat), db / med / 1e6, pf / med / 1e6))
+    # structural check: at fixed (chunk, decode count), latency ~ affine in total KV tokens
+    for c in chunks:
+        for n in decodes:
+            pts = [(r.kv_tokens, r.latency_us) for r in rows if r.chunk == c and r.n_decode == n]
+            if len(pts) >= 3:
+                x = np.array([p[0] for p in pts], dtype=np.float64)
+                y = np.array([p[1] for p in pts], dtype=np.float64)
+                A = np.stack([x, np.ones_like(x)], axis=1)
+                coef, res, _, _ = np.linalg.lstsq(A, y, rcond=None)
+                ss_tot = float(((y - y.mean()) ** 2).sum())
+                r2 = 1.0 - float(((A @ coef - y) ** 2).sum()) / ss_tot if ss_tot > 0 else 1.0
+                print("affine fit chunk=%4d n_dec=%3d: latency_us = %.4g * kv_tokens + %.3g   R^2 = %.4f" % (c, n, coef[0], coef[1], r2))
+    print("%d draws" % len(rows))
+
+
+if __name__ == "__main__":
+    main()
