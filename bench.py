@@ -50,6 +50,27 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel from one ncu capture (see
+# profiles/decode_kernel_config1.md), valid only for the kernel source it was taken on.
+NCU_TRAFFIC = {1: {"decode_cu_sha256_prefix": "f58dfb2a4d4b84bc", "bytes_per_launch": 603.8e6}}
+
+
+def ncu_traffic(workload):
+    """Measured DRAM traffic per launch, or None if the kernel changed since the counters were taken."""
+    import hashlib
+
+    rec = NCU_TRAFFIC.get(workload)
+    if rec is None:
+        return None
+    src = os.path.join(ROOT, "paper_2507_17769_b200", "csrc", "decode.cu")
+    try:
+        with open(src, "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None
+    return rec["bytes_per_launch"] if digest.startswith(rec["decode_cu_sha256_prefix"]) else None
+
+
 class ClockSampler:
     """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
 
@@ -295,7 +316,7 @@ def run_ours(args):
         peaks = measured_peaks()
         achieved = dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else 0.0
         roof = {"kernel": "decode_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
+                "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic(args.workload), "peak_source": peaks["source"],
                 "launch_ms": dec_ms, "algorithmic_bytes_per_launch": dec_bytes, "launches_timed": n_timed}
         pf_tf = pf_flops / (pre_ms * 1e-3) / 1e12 if pf_flops > 0 and pre_ms > 0 else None
         extra = {"decode_kernel_ms": dec_ms, "prefill_kernel_ms": pre_ms, "merge_kernel_ms": mrg_ms,
