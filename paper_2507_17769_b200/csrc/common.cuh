@@ -118,7 +118,7 @@ struct PrefillItem {
     int32_t first_pos;    // absolute position of the tile's first q token (prior + index in chunk)
 };
 
-// Outputs that need the merge kernel: tokens [q_tok, q_tok + n_tok) x heads of
+// Outputs combined from several segments: tokens [q_tok, q_tok + n_tok) x heads of
 // kv head g; partial (i, s, hh) is slot base + s * seg_stride + i * G + hh.
 struct MergeEntry {
     int32_t q_tok;
@@ -135,7 +135,7 @@ struct DeviceWork {       // pointers into the workspace for one run
     const DecodePiece* pieces;
     const DecodeUnit* units;
     const PrefillItem* prefill;
-    const MergeEntry* merge;
+    const MergeEntry* merge;           // prefill q tile pairs cut into segments, combined by the merge kernel
     const DecodeMerge* dmerge;
     int32_t* dmerge_cnt;
     float* part_lse;

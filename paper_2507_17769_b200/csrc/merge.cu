@@ -3,6 +3,9 @@
 // exponential mass: with M = max_s lse_s,
 //     out = sum_s e^{lse_s - M} o_s / sum_s e^{lse_s - M},  lse = M + log sum_s e^{lse_s - M}.
 // Segments are combined in a fixed order, so the result is deterministic.
+// Used for prefill q tile pairs cut into segments: a separate launch spreads the rows over all SMs (letting
+// the last-arriving prefill CTA combine them instead was measured slower: one SM pulls the partial rows
+// too slowly).  Decode rows are combined inside the decode kernel.
 // One warp per output row: the lanes first fetch the row's log-sum-exps in
 // parallel (max and sum by shuffles), then stream the partial rows with several
 // loads in flight.

@@ -31,7 +31,7 @@ struct ps_plan {
     std::vector<DecodePiece> pieces;
     std::vector<DecodeUnit> units;
     std::vector<PrefillItem> prefill;
-    std::vector<MergeEntry> merge;       // combined by the merge kernel (prefill items cut into segments)
+    std::vector<MergeEntry> merge;       // prefill q tile pairs cut into segments: combined by the merge kernel
     std::vector<DecodeMerge> dmerge;     // combined inside the decode kernel
     int64_t decode_merge_rows = 0;
     std::vector<int32_t> prefill_cta_start;  // static partition: CTA b runs items [start[b], start[b+1]); empty = dynamic queue

@@ -41,7 +41,6 @@ constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr int kTileKeys = 128;
 constexpr int kRows = 128;
 constexpr float kRescaleThreshold = 8.f;  // log2 units
-
 // ---- tcgen05 wrappers -------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
@@ -54,6 +53,13 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// One leader lane of a converged warp (always the same one for the full mask).  Issuing the MMAs under this
+// predicate, rather than under a test of the lane index, keeps the descriptor arithmetic warp-uniform.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.b32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -403,6 +409,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                                     float x0, x1, x2, x3;
                                     unpack2(x01, x0, x1);
                                     unpack2(x23, x2, x3);
+                                    // (a cubic on the FMA pipe for part of these was measured slower in every mix)
                                     const float e0 = fast_exp2(x0), e1 = fast_exp2(x1), e2 = fast_exp2(x2), e3 = fast_exp2(x3);
                                     ls0 = add2(ls0, pack2(e0, e1));
                                     ls1 = add2(ls1, pack2(e2, e3));
@@ -555,7 +562,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                         if (!ok) return;
                         tc_fence_after();
                     }
-                    if (lane == 0) {
+                    if (elect_one()) {
                         const uint32_t d_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
                         const uint64_t qd = desc_kmajor + ((sbase + Cfg::kOffQ + x * Cfg::kQBytes) >> 4);
                         const uint64_t kd = desc_kmajor + ((sbase + Cfg::kOffK + s * Cfg::kKBytes) >> 4);
@@ -581,7 +588,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                             if (!ok) break;
                         }
                         tc_fence_after();
-                        if (lane == 0) {
+                        if (elect_one()) {
                             // O_x += P_x V(j): P_x sits in S_x's first 64 columns, two bf16 per column
                             const uint32_t a_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
                             const uint32_t d_addr = tmem + Cfg::kColO + x * Cfg::kColTile;
