@@ -153,6 +153,10 @@ typedef struct {
     int64_t n_partial_slots;   /* fp32 partial rows held in the workspace */
     int64_t total_q_tokens;
     int32_t n_launches;        /* kernels one ps_attn_run launches for this plan */
+    int32_t decode_sms;        /* SMs the decode kernel is sized for */
+    int32_t prefill_sms;       /* SMs the prefill kernel is sized for; in a mixed batch the two kernels run side by
+                                  side on disjoint SMs when that is predicted to be faster (decode_sms + prefill_sms
+                                  = all SMs), otherwise one after the other on all of them */
 } ps_plan_info;
 ps_status ps_plan_get_info(const ps_plan *plan, ps_plan_info *info_out);
 

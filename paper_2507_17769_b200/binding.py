@@ -42,7 +42,8 @@ class ps_plan_opts(ctypes.Structure):
 class ps_plan_info(ctypes.Structure):
     _fields_ = [("n_decode_items", ctypes.c_int32), ("n_prefill_items", ctypes.c_int32), ("n_merge_rows", ctypes.c_int32),
                 ("decode_segment_tokens", ctypes.c_int32), ("prefill_segment_tokens", ctypes.c_int32),
-                ("n_partial_slots", ctypes.c_int64), ("total_q_tokens", ctypes.c_int64), ("n_launches", ctypes.c_int32)]
+                ("n_partial_slots", ctypes.c_int64), ("total_q_tokens", ctypes.c_int64), ("n_launches", ctypes.c_int32),
+                ("decode_sms", ctypes.c_int32), ("prefill_sms", ctypes.c_int32)]
 
 
 class ps_grid_spec(ctypes.Structure):

@@ -157,6 +157,7 @@ struct RunArgs {
     DeviceWork w;
     cudaStream_t stream;
     int num_sms;
+    int dec_sms, pf_sms;  // SMs (= CTAs) for the decode and the prefill kernel
 };
 
 ps_status launch_decode(const RunArgs& a);

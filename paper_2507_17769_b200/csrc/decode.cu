@@ -463,7 +463,7 @@ static ps_status launch_decode_d(const RunArgs& a) {
     p.G = p.Hq / p.Hkv;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
     int grid = (a.w.n_units + kWarps - 1) / kWarps;
-    if (grid > a.num_sms) grid = a.num_sms;
+    if (grid > a.dec_sms) grid = a.dec_sms;
     decode_kernel<D><<<grid, kWarps * 32, Cfg::kSmemBytes, a.stream>>>(p);
     PS_CUDA_TRY(cudaGetLastError());
     return PS_OK;

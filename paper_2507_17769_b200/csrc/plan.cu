@@ -20,6 +20,12 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 constexpr int kDecodeUnitsPerWarp = 1;  // work units per resident warp (measured: 1 beats 2 and 3 on the decode-only batch)
 constexpr int kDecodeMinPages = 8;      // smallest decode unit (pages)
 constexpr int kPrefillKeyTile = 128;    // keys per tensor-core tile
+// Measured on B200 (decode: bandwidth against the number of SMs the kernel runs on; prefill: time of one
+// key-tile step of a q tile pair), used to split the SMs of a mixed batch between the two kernels.
+constexpr double kDecodePeakBytesPerSec = 6.7e12;
+constexpr double kDecodeBytesPerSecPerSm = 125e9;
+constexpr double kPrefillStepSec = 2.5e-6;
+constexpr double kKernelFloorSec = 12e-6;
 
 }  // namespace ps
 
@@ -28,6 +34,11 @@ using namespace ps;
 struct ps_plan {
     ps_shape shape{};
     int32_t n = 0, max_pages = 0, num_sms = 0, device_sms = 0;
+    // SMs given to each kernel: all of them when only one class of rows is present; in a mixed batch the
+    // decode kernel (HBM-bound: a fraction of the SMs saturates the memory system) and the prefill kernel
+    // (tensor-bound) run side by side on disjoint sets of SMs
+    int32_t dec_sms = 0, pf_sms = 0;
+    bool concurrent = false;
     std::vector<DecodePiece> pieces;
     std::vector<DecodeUnit> units;
     std::vector<PrefillItem> prefill;
@@ -50,13 +61,15 @@ struct ps_plan {
     cudaEvent_t ev_copied[2] = {nullptr, nullptr};  // slot's upload finished (copy stream)
     cudaEvent_t ev_done[2] = {nullptr, nullptr};    // the run that used the slot finished (caller's stream)
     cudaEvent_t ev_fence = nullptr;                  // caller's stream position, when the workspace changed
+    cudaStream_t side_stream = nullptr;              // decode kernel of a mixed batch (runs beside the prefill kernel)
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     bool done_valid[2] = {false, false};
     bool copy_pending = false;
     int last_slot = 0;
     unsigned run_no = 0;
     void* last_ws = nullptr;
     WsHeader* last_hdr = nullptr;
-    // optional per-kernel timing: 4 events per recorded run (before prefill, after prefill, after decode, after merge)
+    // optional per-kernel timing: 6 events per recorded run (begin/end of prefill, decode, merge)
     bool timing = false;
     std::vector<cudaEvent_t> tev;
     int timed_runs = 0;
@@ -80,7 +93,7 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
     if (opts && opts->decode_segment_tokens > 0) {
         per_unit = std::max(1, opts->decode_segment_tokens / kPage);
     } else {
-        const int64_t target = (int64_t)pl->num_sms * decode_warps_per_sm() * kDecodeUnitsPerWarp;
+        const int64_t target = (int64_t)pl->dec_sms * decode_warps_per_sm() * kDecodeUnitsPerWarp;
         per_unit = std::max<int64_t>(kDecodeMinPages, (total_pages + target - 1) / target);
     }
     pl->info.decode_segment_tokens = (int32_t)(per_unit * kPage);
@@ -171,13 +184,13 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
                 cuts[i].push_back(kt0);
             }
         }
-    } else if ((int64_t)tiles.size() < 4LL * pl->num_sms) {
+    } else if ((int64_t)tiles.size() < 4LL * pl->pf_sms) {
         // Few items per SM: give every CTA an equal share of the flattened (item, key tile) cost
         // line, cutting items where a share ends.  Only the cut items need the merge.
         static_partition = true;
         double total = 0;
         for (const Tile& t : tiles) total += kPrefillFixedCost + t.key_tiles;
-        const int n_cta = (int)std::max<double>(1, std::min<double>(pl->num_sms, total / kPrefillMinCtaCost));
+        const int n_cta = (int)std::max<double>(1, std::min<double>(pl->pf_sms, total / kPrefillMinCtaCost));
         const double quota = total / n_cta;
         pl->prefill_cta_start.assign(1, 0);
         double cum = 0, boundary = quota;
@@ -309,6 +322,44 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     pl->decode_merge_rows = 0;
     pl->prior.assign(prior_host, prior_host + n);
     pl->info = ps_plan_info{};
+    // ---- split the SMs between the two kernels of a mixed batch ----
+    {
+        double dec_bytes = 0, pf_steps = 0;  // KV bytes the decode rows stream; key-tile steps of the prefill items
+        const int G = shape->n_q_heads / shape->n_kv_heads;
+        const int tile_tok = kPrefillRowsPerItem / G;
+        for (int r = 0; r < n; ++r) {
+            if (q_len_host[r] == 1) {
+                dec_bytes += ((double)prior_host[r] + 1.0) * 2.0 * shape->n_kv_heads * shape->head_dim * 2.0;
+            } else {
+                for (int t0 = 0; t0 < q_len_host[r]; t0 += tile_tok) {
+                    const int n_tok = std::min(tile_tok, q_len_host[r] - t0);
+                    pf_steps += (kPrefillFixedCost + (prior_host[r] + t0 + n_tok + kPrefillKeyTile - 1) / kPrefillKeyTile) * shape->n_kv_heads;
+                }
+            }
+        }
+        pl->dec_sms = pl->pf_sms = pl->num_sms;
+        pl->concurrent = false;
+        if (dec_bytes > 0 && pf_steps > 0 && pl->num_sms >= 16) {
+            // time models (seconds): decode = bytes / min(peak, n * per-SM rate); prefill = steps * step time / m
+            int best_n = 0;
+            double best_t = 1e30;
+            for (int nd = 8; nd <= pl->num_sms - 8; nd += 4) {
+                const double t_dec = dec_bytes / std::min(kDecodePeakBytesPerSec, nd * kDecodeBytesPerSecPerSm) + kKernelFloorSec;
+                const double t_pf = pf_steps * kPrefillStepSec / (pl->num_sms - nd) + kKernelFloorSec;
+                const double t = std::max(t_dec, t_pf);
+                if (t < best_t) {
+                    best_t = t;
+                    best_n = nd;
+                }
+            }
+            const double t_seq = dec_bytes / kDecodePeakBytesPerSec + pf_steps * kPrefillStepSec / pl->num_sms + 2 * kKernelFloorSec;
+            if (best_n > 0 && best_t < 0.95 * t_seq) {
+                pl->dec_sms = best_n;
+                pl->pf_sms = pl->num_sms - best_n;
+                pl->concurrent = true;
+            }
+        }
+    }
     int64_t n_slots = 0;
     plan_decode(pl, prior_host, q_len_host, q_start, opts, &n_slots);
     plan_prefill(pl, prior_host, q_len_host, q_start, opts, &n_slots);
@@ -356,10 +407,15 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
             ok = cudaEventCreateWithFlags(&pl->ev_copied[b], cudaEventDisableTiming) == cudaSuccess &&
                  cudaEventCreateWithFlags(&pl->ev_done[b], cudaEventDisableTiming) == cudaSuccess;
         ok = ok && cudaEventCreateWithFlags(&pl->ev_fence, cudaEventDisableTiming) == cudaSuccess;
+        ok = ok && cudaStreamCreateWithFlags(&pl->side_stream, cudaStreamNonBlocking) == cudaSuccess &&
+             cudaEventCreateWithFlags(&pl->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&pl->ev_join, cudaEventDisableTiming) == cudaSuccess;
         if (!ok) {
             (void)cudaGetLastError();
             if (pl->copy_stream) cudaStreamDestroy(pl->copy_stream);
             pl->copy_stream = nullptr;  // uploads then go on the caller's stream
+            if (pl->side_stream) cudaStreamDestroy(pl->side_stream);
+            pl->side_stream = nullptr;  // mixed batches then run their two kernels one after the other
         }
     }
     memset(pl->pinned, 0, 256);
@@ -381,7 +437,9 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     pl->info.n_merge_rows = (int32_t)merge_rows;
     pl->info.n_partial_slots = n_slots;
     pl->info.total_q_tokens = T;
-    pl->info.n_launches = (pl->units.empty() ? 0 : 1) + (pl->prefill.empty() ? 0 : 1) + (pl->merge.empty() ? 0 : 1);
+    pl->info.decode_sms = pl->dec_sms;
+    pl->info.prefill_sms = pl->pf_sms;
+    pl->info.n_launches = (pl->concurrent && !pl->units.empty() && pl->prefill_cta_start.empty() && (int)pl->prefill.size() > pl->pf_sms ? 1 : 0) + (pl->units.empty() ? 0 : 1) + (pl->prefill.empty() ? 0 : 1) + (pl->merge.empty() ? 0 : 1);
     *plan_inout = pl;
     *workspace_bytes_out = pl->ws_bytes;
     return PS_OK;
@@ -398,6 +456,12 @@ ps_status ps_plan_free(ps_plan* pl) {
         if (pl->ev_done[b]) cudaEventDestroy(pl->ev_done[b]);
     }
     if (pl->ev_fence) cudaEventDestroy(pl->ev_fence);
+    if (pl->side_stream) {
+        cudaStreamSynchronize(pl->side_stream);
+        cudaStreamDestroy(pl->side_stream);
+    }
+    if (pl->ev_fork) cudaEventDestroy(pl->ev_fork);
+    if (pl->ev_join) cudaEventDestroy(pl->ev_join);
     for (cudaEvent_t e : pl->tev) cudaEventDestroy(e);
     if (pl->pinned) { if (pl->pinned_is_cuda) cudaFreeHost(pl->pinned); else free(pl->pinned); }
     delete pl;
@@ -483,6 +547,8 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     a.lse = lse_out_dev;
     a.stream = s;
     a.num_sms = pl->num_sms;
+    a.dec_sms = pl->dec_sms;
+    a.pf_sms = pl->pf_sms;
     a.w.hdr = (WsHeader*)ws;
     a.w.pieces = (const DecodePiece*)(ws + pl->off_pieces);
     a.w.units = (const DecodeUnit*)(ws + pl->off_units);
@@ -498,18 +564,52 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     a.w.prefill_cta_start = (const int32_t*)(ws + pl->off_cta_start);
     a.w.n_prefill_ctas = pl->prefill_cta_start.empty() ? 0 : (int32_t)pl->prefill_cta_start.size() - 1;
 
-    const bool rec = pl->timing && (size_t)(pl->timed_runs + 1) * 4 <= pl->tev.size();
-    cudaEvent_t* ev = rec ? &pl->tev[(size_t)pl->timed_runs * 4] : nullptr;
-    if (rec) cudaEventRecord(ev[0], s);
-    ps_status st = launch_prefill(a);
-    if (st != PS_OK) return st;
-    if (rec) cudaEventRecord(ev[1], s);
-    st = launch_decode(a);
-    if (st != PS_OK) return st;
-    if (rec) cudaEventRecord(ev[2], s);
+    // events per recorded run: prefill begin/end, decode begin/end, merge begin/end
+    const bool rec = pl->timing && (size_t)(pl->timed_runs + 1) * 6 <= pl->tev.size();
+    cudaEvent_t* ev = rec ? &pl->tev[(size_t)pl->timed_runs * 6] : nullptr;
+    ps_status st = PS_OK;
+    if (pl->concurrent && pl->side_stream) {
+        // Mixed batch: the decode kernel runs on its share of the SMs on a second stream while the
+        // prefill kernel runs on the rest.  Both need about 200 KB of shared memory per CTA, so each SM
+        // holds one CTA of either kernel.
+        cudaStream_t side = pl->side_stream;
+        PS_CUDA_TRY(cudaEventRecord(pl->ev_fork, s));
+        PS_CUDA_TRY(cudaStreamWaitEvent(side, pl->ev_fork, 0));
+        if (rec) cudaEventRecord(ev[2], side);
+        RunArgs ad = a;
+        ad.stream = side;
+        st = launch_decode(ad);
+        if (st != PS_OK) return st;
+        if (rec) cudaEventRecord(ev[3], side);
+        if (rec) cudaEventRecord(ev[0], s);
+        st = launch_prefill(a);
+        if (st != PS_OK) return st;
+        if (rec) cudaEventRecord(ev[1], s);
+        if (a.w.n_prefill_ctas == 0 && a.w.n_prefill > a.pf_sms) {
+            // dynamic item queue: once the decode CTAs have left their SMs, as many more prefill CTAs
+            // start there and help drain the same queue
+            RunArgs ah = a;
+            ah.stream = side;
+            ah.pf_sms = a.dec_sms;
+            st = launch_prefill(ah);
+            if (st != PS_OK) return st;
+        }
+        PS_CUDA_TRY(cudaEventRecord(pl->ev_join, side));
+        PS_CUDA_TRY(cudaStreamWaitEvent(s, pl->ev_join, 0));
+    } else {
+        if (rec) cudaEventRecord(ev[0], s);
+        st = launch_prefill(a);
+        if (st != PS_OK) return st;
+        if (rec) cudaEventRecord(ev[1], s);
+        if (rec) cudaEventRecord(ev[2], s);
+        st = launch_decode(a);
+        if (st != PS_OK) return st;
+        if (rec) cudaEventRecord(ev[3], s);
+    }
+    if (rec) cudaEventRecord(ev[4], s);
     st = launch_merge(a);
     if (rec) {
-        cudaEventRecord(ev[3], s);
+        cudaEventRecord(ev[5], s);
         ++pl->timed_runs;
     }
     if (pl->copy_stream && st == PS_OK) {
@@ -524,7 +624,7 @@ ps_status ps_plan_set_timing(ps_plan* pl, int32_t max_runs) {
     if (max_runs < 0 || max_runs > 4096) return fail(PS_ERR_INVALID, "max_runs=%d outside [0, 4096]", max_runs);
     pl->timed_runs = 0;
     pl->timing = max_runs > 0;
-    while (pl->tev.size() < (size_t)max_runs * 4) {
+    while (pl->tev.size() < (size_t)max_runs * 6) {
         cudaEvent_t e;
         PS_CUDA_TRY(cudaEventCreate(&e));
         pl->tev.push_back(e);
@@ -540,7 +640,7 @@ ps_status ps_plan_get_timing(ps_plan* pl, void* stream, float* prefill_ms_out, f
     for (int r = 0; r < pl->timed_runs; ++r)
         for (int k = 0; k < 3; ++k) {
             float ms = 0.f;
-            PS_CUDA_TRY(cudaEventElapsedTime(&ms, pl->tev[(size_t)r * 4 + k], pl->tev[(size_t)r * 4 + k + 1]));
+            PS_CUDA_TRY(cudaEventElapsedTime(&ms, pl->tev[(size_t)r * 6 + 2 * k], pl->tev[(size_t)r * 6 + 2 * k + 1]));
             acc[k] += ms;
         }
     const double n = pl->timed_runs > 0 ? pl->timed_runs : 1;

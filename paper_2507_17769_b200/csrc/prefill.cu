@@ -657,7 +657,7 @@ static ps_status launch_prefill_d(const RunArgs& a) {
     p.Hkv = a.shape.n_kv_heads;
     p.G = p.Hq / p.Hkv;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
-    const int grid = a.w.n_prefill_ctas > 0 ? a.w.n_prefill_ctas : (a.w.n_prefill < a.num_sms ? a.w.n_prefill : a.num_sms);
+    const int grid = a.w.n_prefill_ctas > 0 ? a.w.n_prefill_ctas : (a.w.n_prefill < a.pf_sms ? a.w.n_prefill : a.pf_sms);
     prefill_kernel<D><<<grid, kThreads, Cfg::kSmemBytes, a.stream>>>(p);
     PS_CUDA_TRY(cudaGetLastError());
     return PS_OK;
