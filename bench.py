@@ -175,6 +175,48 @@ def time_oracle(batch, reqs):
     return dt, nbytes, oracle.num_threads()
 
 
+def components_alone(pa, batch, db, out, steps, peaks):
+    """Decode rows alone and prefill rows alone (each on all SMs), for attribution in mixed batches."""
+    import torch
+
+    res = {}
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    q_start = batch.q_start
+    for name, mask in (("decode", batch.q_len == 1), ("prefill", batch.q_len > 1)):
+        idx = np.nonzero(mask)[0]
+        rows = torch.from_numpy(idx).to(db.block_table.device)
+        bt = db.block_table.index_select(0, rows).contiguous()
+        tok = np.concatenate([np.arange(q_start[r], q_start[r] + batch.q_len[r]) for r in idx])
+        q = db.q.index_select(0, torch.from_numpy(tok).to(db.q.device)).contiguous()
+        o = torch.empty_like(q)
+        prior, q_len = batch.prior[idx], batch.q_len[idx]
+
+        def step():
+            pa.plan(prior, q_len, batch.max_pages)
+            pa.run(q, bt, out=o, want_lse=False)
+
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        n = max(3, min(steps, 100))
+        ev0.record()
+        for _ in range(n):
+            step()
+        ev1.record()
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1) / n
+        if name == "decode":
+            res["decode_rows_alone_ms"] = ms
+            res["decode_rows_alone_TBps"] = float(batch.decode_bytes()) / (ms * 1e-3) / 1e12
+        else:
+            tf = float(batch.prefill_flops()) / (ms * 1e-3) / 1e12
+            res["prefill_rows_alone_ms"] = ms
+            res["prefill_rows_alone_TFLOPs"] = tf
+            res["prefill_rows_alone_frac_of_bf16_peak"] = tf / peaks["bf16_tflops"]
+    pa.plan(batch.prior, batch.q_len, batch.max_pages)  # back to the full batch
+    return res
+
+
 def run_reference(args):
     rank, _, _ = dist_env()
     if rank != 0:
@@ -322,7 +364,12 @@ def run_ours(args):
         extra = {"decode_kernel_ms": dec_ms, "prefill_kernel_ms": pre_ms, "merge_kernel_ms": mrg_ms,
                  "decode_TBps_kernel": achieved / 1e3, "prefill_TFLOPs_kernel": pf_tf,
                  "prefill_frac_of_bf16_peak": pf_tf / peaks["bf16_tflops"] if pf_tf else None,
-                 "value_frac_of_nominal_8TBps": value / world / 8.0, "host_issue_ms_per_step": host_ms}
+                 "value_frac_of_nominal_8TBps": value / world / 8.0, "host_issue_ms_per_step": host_ms,
+                 "decode_sms": info.decode_sms, "prefill_sms": info.prefill_sms,
+                 "side_by_side": bool(pf_flops > 0 and dec_bytes > 0 and info.decode_sms + info.prefill_sms <= 148
+                                      and info.decode_sms != info.prefill_sms)}
+        if pf_flops > 0 and dec_bytes > 0:
+            extra.update(components_alone(pa, batch, db, out, args.steps, peaks))
         line = {
             "metric": METRIC, "value": value, "unit": "TB/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",

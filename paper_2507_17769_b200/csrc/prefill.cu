@@ -217,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
             mbar_init(bars + Bars::v_full + 8 * s, 1);
             mbar_init(bars + Bars::v_empty + 8 * s, 1);
             mbar_init(bars + Bars::s_full + 8 * s, 1);
-            mbar_init(bars + Bars::p_ready + 8 * s, kRows);
+            mbar_init(bars + Bars::p_ready + 8 * s, kRows / 32);
             mbar_init(bars + Bars::o_done + 8 * s, 1);
         }
         mbar_fence_init();
@@ -445,7 +445,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                         fence_proxy_async_smem();
                     }
                     tc_fence_before();
-                    mbar_arrive(bars + Bars::p_ready + 8 * x);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bars + Bars::p_ready + 8 * x);  // one arrival per softmax warp
                 }
                 // ---- epilogue: O / l ----
                 if (ok) ok = wait_all(bars + Bars::o_done + 8 * x, (x ? item_ctr_b : item_ctr) & 1, s_abort);
