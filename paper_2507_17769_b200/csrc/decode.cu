@@ -100,9 +100,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
     auto produce = [&]() {
         while (!P_done && P_page >= P_page_end) {
             if (++P_piece >= P_piece_end) {
-                int u = 0;
-                if (lane == 0) u = atomicAdd(&p.hdr->decode_next, 1);
-                u = __shfl_sync(0xffffffffu, u, 0);
+                // a warp's first unit is its own index (no round trip); later ones come from the shared counter
+                int u = blockIdx.x * kWarps + warp;
+                if (pseq > 0) {
+                    if (lane == 0) u = atomicAdd(&p.hdr->decode_next, 1) + gridDim.x * kWarps;
+                    u = __shfl_sync(0xffffffffu, u, 0);
+                }
                 if (lane == 0) ring[pseq % kRing] = u;
                 ++pseq;
                 if (u >= p.n_units) { P_done = true; break; }
