@@ -168,3 +168,23 @@ def test_decode_units_are_balanced():
     # partial rows stay a small fraction of the KV stream
     assert info.n_partial_slots * 128 * 4 < 0.1 * b.decode_bytes()
     ps.ps_plan_free(plan)
+
+
+def test_mixed_batches_split_the_sms_and_single_class_batches_do_not():
+    sh = ps.make_shape(32, 8, 128)
+    for make, mixed in [(gen.config1, False), (gen.config2, True), (lambda: gen.make_batch(gen.SHAPE_8B, 5, [700], [300]), False),
+                        (lambda: gen.config3_cell(64, 8, 512, 3000), True)]:
+        b = make()
+        plan, _ = ps.ps_attn_plan(sh, b.prior, b.q_len, b.max_pages, opts())
+        info = ps.ps_plan_get_info(plan)
+        if mixed:
+            assert info.decode_sms + info.prefill_sms == 148 and info.decode_sms >= 8 and info.prefill_sms >= 8
+        else:
+            assert info.decode_sms == 148 and info.prefill_sms == 148
+        coverage_check(b, plan)
+        ps.ps_plan_free(plan)
+    big = gen.config4()
+    plan, _ = ps.ps_attn_plan(ps.make_shape(64, 8, 128), big.prior, big.q_len, big.max_pages, opts())
+    info = ps.ps_plan_get_info(plan)
+    assert info.decode_sms + info.prefill_sms == 148 and info.prefill_sms > info.decode_sms  # prefill-heavy batch
+    ps.ps_plan_free(plan)

@@ -157,9 +157,18 @@ def chunk_sample(c):
 
 
 def test_config2_mixed_batch_sampled_parity():
+    import torch
+
     b = gen.config2()
     dec = [0, 1, int(np.argmax(b.kv_len[:512])), int(np.argmin(b.kv_len[:512]))]
-    sampled_parity(b, dec, {512: chunk_sample(1536)}, "config2")
+    _, db = sampled_parity(b, dec, {512: chunk_sample(1536)}, "config2")
+    # the two kernels of this batch run side by side on disjoint SMs; the result is still the same bits every run
+    info = db.plan()
+    assert 0 < info.decode_sms < info.decode_sms + info.prefill_sms and info.decode_sms != info.prefill_sms
+    o1, l1 = db.run()
+    o2, l2 = db.run()
+    db.pa.check()
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)
 
 
 def test_config3_cells_sampled_parity():
