@@ -124,7 +124,8 @@ ps_status ps_kv_status(ps_kv *kv, void *stream);
  * Partition one batch into work items.  Rows with q_len == 1 are decode rows
  * (memory-bound KV streaming, section 2.2); rows with q_len > 1 are prefill
  * chunks (dense contraction, section 3.4).  Long contexts are cut into KV
- * segments whose partial results a merge kernel combines.  Host arrays
+ * segments whose partial results are combined afterwards (decode rows inside
+ * the decode kernel, prefill items by a merge kernel).  Host arrays
  * prior_host / q_len_host have n entries and are read before the call returns.
  * max_pages_per_seq is the row stride of the block table later given to
  * ps_attn_run; kv_len[r] must not exceed max_pages_per_seq * page_size.
@@ -147,7 +148,7 @@ ps_status ps_plan_free(ps_plan *plan);
 typedef struct {
     int32_t n_decode_items;
     int32_t n_prefill_items;
-    int32_t n_merge_rows;      /* (token, q head) outputs that need the merge kernel */
+    int32_t n_merge_rows;      /* (token, q head) outputs combined from several KV segments */
     int32_t decode_segment_tokens;
     int32_t prefill_segment_tokens;
     int64_t n_partial_slots;   /* fp32 partial rows held in the workspace */
@@ -189,7 +190,10 @@ ps_status ps_plan_get_items(const ps_plan *plan, int32_t *decode_items_out, int6
  * the work list is uploaded (on a stream of the plan's own, ordered against
  * `stream` with events, into one of two slots of the workspace so that it can
  * run under the previous run's kernels), then the prefill, decode and merge
- * kernels run on `stream`.  Consecutive runs of one plan must be issued to the
+ * kernels run; for a batch with both row classes the decode kernel may run on
+ * a second stream of the plan, beside the prefill kernel on disjoint SMs, and
+ * is joined back into `stream` before the call's work is complete in stream
+ * order.  Consecutive runs of one plan must be issued to the
  * same stream, or be ordered by the caller: they share the partial buffers.
  * Returns host-detectable errors only (PS_ERR_INVALID, PS_ERR_WORKSPACE,
  * PS_ERR_CUDA); errors seen on the device are read with ps_plan_status.
@@ -240,8 +244,10 @@ ps_status ps_attn_run_static(ps_plan *plan, const ps_kv *kv, const void *q_dev, 
  * Per-kernel timing of the next runs of this plan (the profile of section 4.5
  * split into its prefill-attention and decode-attention terms, section 3.4).
  * ps_plan_set_timing(plan, max_runs) makes each of the next max_runs calls of
- * ps_attn_run record CUDA events on its stream around the prefill, decode and
- * merge launches (max_runs = 0 switches recording off); calling it again
+ * ps_attn_run record CUDA events around the prefill, decode and merge launches
+ * (on the stream each is launched on; max_runs = 0 switches recording off;
+ * when the two kernels of a mixed batch run side by side their intervals
+ * overlap and each is longer than the kernel would take alone); calling it again
  * restarts the count.  ps_plan_get_timing synchronises `stream` and returns
  * the mean duration in milliseconds of each kernel over the runs recorded so
  * far, and how many there were.  A kernel the plan does not launch reports the

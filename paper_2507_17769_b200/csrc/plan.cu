@@ -4,7 +4,6 @@
 // batch produces the same items, the same summation order and therefore the
 // same output bits under any assignment of physical pages.
 #include <algorithm>
-#include <chrono>
 #include <cstdlib>
 #include <cmath>
 #include <cstring>
