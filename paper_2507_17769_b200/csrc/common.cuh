@@ -158,6 +158,7 @@ struct RunArgs {
     cudaStream_t stream;
     int num_sms;
     int dec_sms, pf_sms;  // SMs (= CTAs) for the decode and the prefill kernel
+    int32_t total_q;      // q tokens of the batch (rows of q and out)
 };
 
 ps_status launch_decode(const RunArgs& a);

@@ -548,6 +548,7 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     a.num_sms = pl->num_sms;
     a.dec_sms = pl->dec_sms;
     a.pf_sms = pl->pf_sms;
+    a.total_q = pl->info.total_q_tokens;
     a.w.hdr = (WsHeader*)ws;
     a.w.pieces = (const DecodePiece*)(ws + pl->off_pieces);
     a.w.units = (const DecodeUnit*)(ws + pl->off_units);

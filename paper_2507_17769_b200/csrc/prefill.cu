@@ -5,26 +5,36 @@
 // bound (section 3.4), so QK^T and PV run as tcgen05.mma with fp32
 // accumulators in tensor memory.
 //
-// One CTA works on one item = up to two consecutive q tiles (A, B) of 128
-// (token, head) rows each -- the G heads that share a kv head x 128 / G
-// consecutive tokens -- over one key range.  Both tiles consume the same K and V
-// tiles from shared memory, and while one tile's softmax runs on the CUDA cores
-// the tensor core works for the other tile (ping-pong).
+// One CTA works through a list of items; an item = up to two consecutive q tiles
+// (A, B) of 128 (token, head) rows each -- the G heads that share a kv head x
+// 128 / G consecutive tokens -- over one key range.  Both tiles consume the same
+// K and V tiles from shared memory, and while one tile's softmax runs on the
+// CUDA cores the tensor core works for the other tile (ping-pong).
 //
 //   warps 0-3  softmax of tile A: thread t owns row t (= TMEM lane t); one
 //              tcgen05.ld pass over S, causal mask by prior + i, running max
 //              with lazy rescaling of O, P (bf16) stored back into the TMEM
-//              columns S occupied, O / l and the log-sum-exp at the end
+//              columns S occupied; at the end of the item O / l and the
+//              log-sum-exp, transposed through shared memory so that global
+//              stores cover whole rows
 //   warps 4-7  the same for tile B
-//   warp 8     producer: one 2 KB bulk async copy per (page, K|V, d half) into
-//              2-stage K and V rings; the pool's page layout already is the
+//   warp 8     producer: fetches the CTA's next item and publishes its record in
+//              a shared-memory ring; Q tiles by tensor-map loads (128-byte
+//              swizzle); one 2 KB bulk async copy per (page, K|V, d half) into
+//              2-stage K and V rings -- the pool's page layout already is the
 //              128-byte-swizzled operand layout, so blocks are consumed in place
 //   warp 9     MMA issue: S_X = Q_X K^T (SS form, M128 N128 K16) and
 //              O_X += P_X V (A operand from TMEM, V as MN-major B operand,
 //              M128 N=d K16); completion signalled with tcgen05.commit
 //
+// The roles synchronise through mbarriers only, so consecutive items overlap:
+// the next item's Q, first K/V tiles and first QK^T are under way while the
+// current item's last softmax, PV and output are still running.
+//
 // TMEM columns: S_A 0..127, S_B 128..255, O_A 256.., O_B 384.. (512 allocated).
 // Every wait is bounded; on expiry the CTA sets the timeout status and drains.
+#include <cuda.h>
+
 #include "common.cuh"
 
 namespace ps {
@@ -33,10 +43,10 @@ namespace {
 
 constexpr int kSoftmaxThreads = 256;
 // Three warpgroups: two of softmax warps and one holding the producer and MMA warps (its
-// other two warps only take part in the CTA-wide barriers).  Registers are re-split after
-// start-up: 384 threads x 168 at launch = 2 x 128 x 200 + 128 x 104.
+// other two warps have no work).  Registers are re-split after
+// start-up: 384 threads x 168 at launch = 2 x 128 x 192 + 128 x 120.
 constexpr int kThreads = kSoftmaxThreads + 128;
-constexpr int kRegsSoftmax = 200, kRegsOther = 104;
+constexpr int kRegsSoftmax = 192, kRegsOther = 120;
 constexpr int kProducerWarp = 8, kMmaWarp = 9;
 constexpr int kTileKeys = 128;
 constexpr int kRows = 128;
@@ -126,6 +136,13 @@ __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+// One box of a 3-d tensor map into shared memory; completion is counted in bytes on `bar`.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -145,6 +162,8 @@ __host__ __device__ constexpr uint32_t instr_desc(int n, bool b_mn_major) {
            ((uint32_t)(kRows >> 4) << 24);
 }
 
+constexpr int kBarBlockBytes = 512;  // mbarriers, flags and the item record ring
+
 template <int D>
 struct PrefillCfg {
     static constexpr int kHalves = D / 64;
@@ -156,8 +175,10 @@ struct PrefillCfg {
     static constexpr int kOffQ = 0;                              // Q_A, Q_B
     static constexpr int kOffK = kOffQ + 2 * kQBytes;
     static constexpr int kOffV = kOffK + kStages * kKBytes;
-    static constexpr int kOffBar = kOffV + kStages * kVBytes;
-    static constexpr int kSmemBytes = kOffBar + 256 + 1024;      // + alignment slack
+    static constexpr int kStageWarpBytes = 32 * 128;             // output staging: 32 rows x 128 bytes per softmax warp
+    static constexpr int kOffStage = kOffV + kStages * kVBytes;
+    static constexpr int kOffBar = kOffStage + 8 * kStageWarpBytes;
+    static constexpr int kSmemBytes = kOffBar + kBarBlockBytes + 1024;  // + alignment slack
     static constexpr int kTmemCols = 512;
     static constexpr uint32_t kColS = 0, kColO = 256, kColTile = 128;  // tile X at + X * 128
 };
@@ -165,7 +186,6 @@ struct PrefillCfg {
 struct PrefillParams {
     const char* pool;
     int64_t num_pages;
-    const __nv_bfloat16* q;
     const int32_t* block_table;
     int32_t max_pages;
     __nv_bfloat16* out;
@@ -180,10 +200,17 @@ struct PrefillParams {
     float scale_log2;
 };
 
-struct Bars {  // byte offsets from the barrier block; [2] = one per stage or per tile
+constexpr int kItemRing = 4;        // item records in flight between the producer and the other roles
+constexpr int kConsumerWarps = 9;   // eight softmax warps and the MMA warp read every record
+
+struct Bars {  // byte offsets from the barrier block; [2] = one per stage or per q tile
     static constexpr int k_full = 0, k_empty = 16, v_full = 32, v_empty = 48, s_full = 64, p_ready = 80, o_done = 96;
-    static constexpr int tmem_slot = 112, item_slot = 116, abort_slot = 120;
+    static constexpr int q_full = 112, q_empty = 128, item_full = 144, item_empty = item_full + 8 * kItemRing;
+    static constexpr int tmem_slot = item_empty + 8 * kItemRing, abort_slot = tmem_slot + 4;
+    static constexpr int ring = 256;  // kItemRing PrefillItem records
+    static constexpr int bytes = ring + kItemRing * (int)sizeof(PrefillItem);
 };
+static_assert(Bars::abort_slot + 4 <= Bars::ring && sizeof(PrefillItem) == 32 && Bars::bytes <= kBarBlockBytes, "barrier block layout");
 
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
     for (uint32_t i = 0; i < 40000000u; ++i) {
@@ -199,15 +226,15 @@ __device__ __forceinline__ bool wait_all(uint32_t bar, uint32_t parity, volatile
 }
 
 template <int D>
-__global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParams p) {
+__global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap q_map) {
     using Cfg = PrefillCfg<D>;
     extern __shared__ char smem_raw[];
     char* smem = reinterpret_cast<char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t sbase = smem_u32(smem);
     const uint32_t bars = sbase + Cfg::kOffBar;
     volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + Cfg::kOffBar + Bars::tmem_slot);
-    volatile int* s_item = reinterpret_cast<volatile int*>(smem + Cfg::kOffBar + Bars::item_slot);
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Cfg::kOffBar + Bars::abort_slot);
+    uint4* ring = reinterpret_cast<uint4*>(smem + Cfg::kOffBar + Bars::ring);  // two uint4 per record
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -219,6 +246,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
             mbar_init(bars + Bars::s_full + 8 * s, 1);
             mbar_init(bars + Bars::p_ready + 8 * s, kRows / 32);
             mbar_init(bars + Bars::o_done + 8 * s, 1);
+            mbar_init(bars + Bars::q_full + 8 * s, 1);
+            mbar_init(bars + Bars::q_empty + 8 * s, 1);
+        }
+        for (int s = 0; s < kItemRing; ++s) {
+            mbar_init(bars + Bars::item_full + 8 * s, 1);
+            mbar_init(bars + Bars::item_empty + 8 * s, kConsumerWarps);
         }
         mbar_fence_init();
         *s_abort = 0;
@@ -232,44 +265,28 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
     tc_fence_after();
     const uint32_t tmem = (uint32_t)*s_tmem;
 
-    // Phase counters; every role advances them identically.  Tile B's barriers only move in
-    // items that have a second q tile, so they are counted separately.
-    uint32_t tile_ctr = 0, tile_ctr_b = 0;  // key tiles processed so far (all items / items with a tile B)
-    uint32_t item_ctr = 0, item_ctr_b = 0;  // items processed (phase of the per-item o_done barriers)
+    // The roles never meet at a CTA-wide barrier after this point: items flow through the record ring
+    // and the mbarriers, so the next item's Q, K and first QK^T overlap the current item's last
+    // softmax, PV and output.  Every role counts items and key tiles identically to derive barrier
+    // phases; tile B's barriers only move in items that have a second q tile.
     constexpr uint32_t kIdescQK = instr_desc(kTileKeys, false);
     constexpr uint32_t kIdescPV = instr_desc(D, true);
     static_assert(kPrefillRowsPerItem == 2 * kRows, "the planner pairs two q tiles per item");
     const int tile_tok = kRows / p.G;
+    const int g_shift = 31 - __clz(p.G);  // G is a power of two
 
-    // Every role runs this at the top of each item; two CTA-wide barriers per item (after the
-    // item fetch, after the Q tiles are in shared memory) are executed by all 12 warps.
-    PrefillItem it;
-    int n_tiles = 0;
-    bool has_b = false;
-    int static_cur = p.cta_start ? p.cta_start[blockIdx.x] : 0;
-    const int static_end = p.cta_start ? p.cta_start[blockIdx.x + 1] : 0;
-    auto next_item = [&]() -> bool {
-        if (threadIdx.x == 0)
-            *s_item = p.cta_start ? (static_cur < static_end ? static_cur : p.n_items) : atomicAdd(&p.hdr->prefill_next, 1);
-        ++static_cur;
-        tc_fence_before();
-        __syncthreads();
-        tc_fence_after();
-        const int item_idx = *s_item;
-        if (item_idx >= p.n_items || *s_abort) return false;
-        it = p.items[item_idx];
-        n_tiles = (it.key_end - it.key_begin + kTileKeys - 1) / kTileKeys;
-        has_b = it.n_tok > tile_tok;
-        return true;
+    // consumer side of the record ring: record number n into `it`; false at the end-of-work record or on abort
+    auto take_item = [&](uint32_t n, PrefillItem& it) -> bool {
+        const uint32_t slot = n % kItemRing;
+        if (!wait_all(bars + Bars::item_full + 8 * slot, (n / kItemRing) & 1, s_abort)) return false;
+        const uint4 a = ring[2 * slot], b = ring[2 * slot + 1];
+        it.req = (int32_t)a.x, it.kv_head = (int32_t)a.y, it.key_begin = (int32_t)a.z, it.key_end = (int32_t)a.w;
+        it.q_tok = (int32_t)b.x, it.n_tok = (int32_t)b.y, it.part_slot = (int32_t)b.z, it.first_pos = (int32_t)b.w;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + Bars::item_empty + 8 * slot);
+        return it.n_tok > 0;
     };
-    auto advance = [&]() {
-        tile_ctr += n_tiles;
-        ++item_ctr;
-        if (has_b) {
-            tile_ctr_b += n_tiles;
-            ++item_ctr_b;
-        }
-    };
+    auto tiles_of = [](const PrefillItem& it) { return (it.key_end - it.key_begin + kTileKeys - 1) / kTileKeys; };
 
     if (warp < 8) {
         // ====================================================================
@@ -280,33 +297,24 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t s_addr = tmem + lane_addr + Cfg::kColS + x * Cfg::kColTile;
         const uint32_t o_addr = tmem + lane_addr + Cfg::kColO + x * Cfg::kColTile;
-        const int hh = t % p.G;
-        while (next_item()) {
-            // ---- Q tile x -> shared memory (row t = token x * tile_tok + t / G, head t % G) ----
-            const int i = x * tile_tok + t / p.G;
-            const bool valid = i < it.n_tok;
-            {
-                const uint4* src = reinterpret_cast<const uint4*>(
-                    p.q + ((int64_t)(it.q_tok + (valid ? i : 0)) * p.Hq + it.kv_head * p.G + hh) * D);
-                char* qdst = smem + Cfg::kOffQ + x * Cfg::kQBytes + t * 128;
-#pragma unroll
-                for (int U = 0; U < D / 8; ++U) {
-                    const uint4 v = valid ? __ldg(src + U) : make_uint4(0, 0, 0, 0);
-                    *reinterpret_cast<uint4*>(qdst + (U >> 3) * Cfg::kHalfBytes + (((U & 7) ^ (t & 7)) << 4)) = v;
-                }
-                fence_proxy_async_smem();
-            }
-            __syncthreads();
-
+        const int hh = t & (p.G - 1);
+        char* const stg = smem + Cfg::kOffStage + warp * Cfg::kStageWarpBytes;
+        uint32_t n_item = 0, tile_ctr = 0, tiles_x = 0, items_x = 0;
+        PrefillItem it;
+        bool ok = true;
+        while (ok && take_item(n_item, it)) {
+            ++n_item;
+            const int n_tiles = tiles_of(it);
+            const bool has_b = it.n_tok > tile_tok;
             if (x == 0 || has_b) {
-                const int limit = it.first_pos + i;  // last visible key of this row
+                const int i = x * tile_tok + (t >> g_shift);  // token of this row within the item
+                const bool valid = i < it.n_tok;               // rows past the chunk's end compute on whatever the Q load brought
+                const int limit = it.first_pos + i;            // last visible key of this row
                 const int tile_first_pos = it.first_pos + x * tile_tok;
                 float m = -INFINITY, l = 0.f;
-                bool ok = true;
                 for (int j = 0; j < n_tiles && ok; ++j) {
-                    const uint32_t tc = tile_ctr + j;                          // K/V stage phase
-                    const uint32_t tcx = (x ? tile_ctr_b : tile_ctr) + j;     // phase of this tile's own barriers
-                    ok = wait_all(bars + Bars::s_full + 8 * x, tcx & 1, s_abort);
+                    const uint32_t tc = tile_ctr + j;  // K/V stage phase
+                    ok = wait_all(bars + Bars::s_full + 8 * x, (tiles_x + j) & 1, s_abort);
                     if (!ok) break;
                     tc_fence_after();
                     const int tile_base = it.key_begin + j * kTileKeys;
@@ -448,64 +456,119 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                     __syncwarp();
                     if (lane == 0) mbar_arrive(bars + Bars::p_ready + 8 * x);  // one arrival per softmax warp
                 }
-                // ---- epilogue: O / l ----
-                if (ok) ok = wait_all(bars + Bars::o_done + 8 * x, (x ? item_ctr_b : item_ctr) & 1, s_abort);
+                // ---- output: O / l through this warp's staging slice, so that global stores cover whole rows ----
+                if (ok) ok = wait_all(bars + Bars::o_done + 8 * x, items_x & 1, s_abort);
                 if (ok) {
                     tc_fence_after();
                     const float inv = l > 0.f ? 1.f / l : 0.f;
                     const float lse_v = l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -INFINITY;
-                    const int64_t orow = (int64_t)(it.q_tok + i) * p.Hq + it.kv_head * p.G + hh;
-                    const int64_t prow = (int64_t)it.part_slot + (int64_t)i * p.G + hh;
+                    const int row0 = (warp & 3) * 32;          // first tile row of this warp
+                    const int sub = lane >> 3, unit = lane & 7;  // write-out: 4 rows per instruction, 8 lanes x 16 bytes per row
+                    char* const my_row = stg + lane * 128;
+                    if (it.part_slot < 0) {
+                        // final output: bf16, 64 columns (128 bytes of each row) per pass
 #pragma unroll 1
-                    for (int c0 = 0; c0 < D; c0 += 32) {
-                        uint32_t v[32];
-                        tmem_ld32(o_addr + c0, v);
-                        tmem_wait_ld();
-                        if (!valid) continue;
-                        if (it.part_slot < 0) {
-                            uint4* dst = reinterpret_cast<uint4*>(p.out + orow * D + c0);
+                        for (int c0 = 0; c0 < D; c0 += 64) {
+                            uint32_t v[2][32];
+                            tmem_ld32(o_addr + c0, v[0]);
+                            tmem_ld32(o_addr + c0 + 32, v[1]);
+                            tmem_wait_ld();
 #pragma unroll
-                            for (int u = 0; u < 4; ++u) {
+                            for (int u = 0; u < 8; ++u) {
+                                const uint32_t* s = &v[u >> 2][(u & 3) * 8];
                                 uint4 w;
-                                w.x = pack_bf16(__uint_as_float(v[8 * u + 0]) * inv, __uint_as_float(v[8 * u + 1]) * inv);
-                                w.y = pack_bf16(__uint_as_float(v[8 * u + 2]) * inv, __uint_as_float(v[8 * u + 3]) * inv);
-                                w.z = pack_bf16(__uint_as_float(v[8 * u + 4]) * inv, __uint_as_float(v[8 * u + 5]) * inv);
-                                w.w = pack_bf16(__uint_as_float(v[8 * u + 6]) * inv, __uint_as_float(v[8 * u + 7]) * inv);
-                                dst[u] = w;
+                                w.x = pack_bf16(__uint_as_float(s[0]) * inv, __uint_as_float(s[1]) * inv);
+                                w.y = pack_bf16(__uint_as_float(s[2]) * inv, __uint_as_float(s[3]) * inv);
+                                w.z = pack_bf16(__uint_as_float(s[4]) * inv, __uint_as_float(s[5]) * inv);
+                                w.w = pack_bf16(__uint_as_float(s[6]) * inv, __uint_as_float(s[7]) * inv);
+                                *reinterpret_cast<uint4*>(my_row + ((u ^ (lane & 7)) << 4)) = w;
                             }
-                        } else {
-                            float4* dst = reinterpret_cast<float4*>(p.part_o + prow * D + c0);
+                            __syncwarp();
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const int r = k * 4 + sub, tt = row0 + r;
+                                const int i_r = x * tile_tok + (tt >> g_shift);
+                                if (i_r < it.n_tok) {
+                                    const uint4 w = *reinterpret_cast<const uint4*>(stg + r * 128 + ((unit ^ (r & 7)) << 4));
+                                    const int64_t orow_r = (int64_t)(it.q_tok + i_r) * p.Hq + it.kv_head * p.G + (tt & (p.G - 1));
+                                    *reinterpret_cast<uint4*>(p.out + orow_r * D + c0 + unit * 8) = w;
+                                }
+                            }
+                            __syncwarp();
+                        }
+                        if (valid && p.lse) p.lse[(int64_t)(it.q_tok + i) * p.Hq + it.kv_head * p.G + hh] = lse_v;
+                    } else {
+                        // partial result of a cut item: fp32 rows at consecutive slots, 32 columns per pass
+                        const int64_t prow0 = (int64_t)it.part_slot + x * kRows + row0;
+#pragma unroll 1
+                        for (int c0 = 0; c0 < D; c0 += 32) {
+                            uint32_t v[32];
+                            tmem_ld32(o_addr + c0, v);
+                            tmem_wait_ld();
 #pragma unroll
                             for (int u = 0; u < 8; ++u)
-                                dst[u] = make_float4(__uint_as_float(v[4 * u]) * inv, __uint_as_float(v[4 * u + 1]) * inv,
-                                                     __uint_as_float(v[4 * u + 2]) * inv, __uint_as_float(v[4 * u + 3]) * inv);
+                                *reinterpret_cast<float4*>(my_row + ((u ^ (lane & 7)) << 4)) =
+                                    make_float4(__uint_as_float(v[4 * u]) * inv, __uint_as_float(v[4 * u + 1]) * inv,
+                                                __uint_as_float(v[4 * u + 2]) * inv, __uint_as_float(v[4 * u + 3]) * inv);
+                            __syncwarp();
+#pragma unroll
+                            for (int k = 0; k < 8; ++k) {
+                                const int r = k * 4 + sub, tt = row0 + r;
+                                if (x * tile_tok + (tt >> g_shift) < it.n_tok)
+                                    *reinterpret_cast<float4*>(p.part_o + (prow0 + r) * D + c0 + unit * 4) =
+                                        *reinterpret_cast<const float4*>(stg + r * 128 + ((unit ^ (r & 7)) << 4));
+                            }
+                            __syncwarp();
                         }
-                    }
-                    if (valid) {
-                        if (it.part_slot < 0) {
-                            if (p.lse) p.lse[orow] = lse_v;
-                        } else {
-                            p.part_lse[prow] = lse_v;
-                        }
+                        if (valid) p.part_lse[prow0 + lane] = lse_v;
                     }
                 }
+                tiles_x += n_tiles;
+                ++items_x;
             }
-            advance();
+            tile_ctr += n_tiles;
         }
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsOther));
         if (warp == kProducerWarp) {
             // ================================================================
-            // producer
+            // producer: item records, Q tiles (tensor-map loads), K and V tiles (bulk copies of pool blocks)
             // ================================================================
             const int pg = lane >> 2, which = lane & 3;  // page in tile; 0/1 = K half 0/1, 2/3 = V half 0/1
             constexpr uint32_t kPieceBytes = kPage * 128;  // 16 tokens x 64 elements
-            while (next_item()) {
-                // K and V do not depend on the Q tiles: the first tile's copies are issued before this
-                // warp joins the item's second CTA-wide barrier (Q tiles in shared memory)
-                bool joined = false;
+            uint32_t n_item = 0, tile_ctr = 0, items_x[2] = {0, 0};
+            int static_cur = p.cta_start ? p.cta_start[blockIdx.x] : 0;
+            const int static_end = p.cta_start ? p.cta_start[blockIdx.x + 1] : 0;
+            bool ok = true;
+            while (ok) {
+                // next item of this CTA's static share, or of the queue all CTAs of the run drain
+                int idx = 0;
+                if (lane == 0)
+                    idx = p.cta_start ? (static_cur < static_end ? static_cur : p.n_items) : atomicAdd(&p.hdr->prefill_next, 1);
+                ++static_cur;
+                idx = __shfl_sync(0xffffffffu, idx, 0);
+                uint4 rec0 = make_uint4(0, 0, 0, 0), rec1 = make_uint4(0, 0, 0, 0);  // n_tok = 0: end of work
+                if (idx < p.n_items) {
+                    const uint4* src = reinterpret_cast<const uint4*>(p.items + idx);
+                    rec0 = __ldg(src);
+                    rec1 = __ldg(src + 1);
+                }
+                const uint32_t slot = n_item % kItemRing;
+                ok = wait_all(bars + Bars::item_empty + 8 * slot, ((n_item / kItemRing) & 1) ^ 1, s_abort);
+                if (!ok) break;
+                if (lane == 0) {
+                    ring[2 * slot] = rec0;
+                    ring[2 * slot + 1] = rec1;
+                    mbar_arrive(bars + Bars::item_full + 8 * slot);
+                }
+                ++n_item;
+                PrefillItem it;
+                it.req = (int32_t)rec0.x, it.kv_head = (int32_t)rec0.y, it.key_begin = (int32_t)rec0.z, it.key_end = (int32_t)rec0.w;
+                it.q_tok = (int32_t)rec1.x, it.n_tok = (int32_t)rec1.y, it.part_slot = (int32_t)rec1.z, it.first_pos = (int32_t)rec1.w;
+                if (it.n_tok <= 0) break;
+                const int n_tiles = tiles_of(it);
+                const int n_x = it.n_tok > tile_tok ? 2 : 1;
                 const int32_t* bt = p.block_table + (int64_t)it.req * p.max_pages + it.key_begin / kPage;
-                bool ok = true;
                 for (int j = 0; j < n_tiles && ok; ++j) {
                     const uint32_t tc = tile_ctr + j;
                     const uint32_t s = tc & 1, par = (tc >> 1) & 1;
@@ -528,6 +591,26 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                         bulk_g2s(sbase + Cfg::kOffK + s * Cfg::kKBytes + which * Cfg::kHalfBytes + pg * kPieceBytes,
                                  src + which * kPieceBytes, kPieceBytes, bars + Bars::k_full + 8 * s);
 
+                    if (j == 0) {
+                        // Q tile x: rows (token, head of the group) in token-major order, one box of
+                        // [128 / G tokens][G heads][64 elements] per 64-element half, written with the
+                        // 128-byte swizzle the MMA descriptors expect.  The buffer is free once the
+                        // previous item's last QK^T of that tile has run.
+                        for (int x = 0; x < n_x && ok; ++x) {
+                            ok = wait_all(bars + Bars::q_empty + 8 * x, (items_x[x] & 1) ^ 1, s_abort);
+                            if (!ok) break;
+                            if (lane == 0) {
+                                mbar_expect_tx(bars + Bars::q_full + 8 * x, Cfg::kQBytes);
+#pragma unroll
+                                for (int h = 0; h < Cfg::kHalves; ++h)
+                                    tma_load_3d(sbase + Cfg::kOffQ + x * Cfg::kQBytes + h * Cfg::kHalfBytes, &q_map, h * 64,
+                                                it.kv_head * p.G, it.q_tok + x * tile_tok, bars + Bars::q_full + 8 * x);
+                            }
+                            __syncwarp();
+                        }
+                        if (!ok) break;
+                    }
+
                     ok = wait_all(bars + Bars::v_empty + 8 * s, par ^ 1, s_abort);
                     if (!ok) break;
                     if (lane == 0) mbar_expect_tx(bars + Bars::v_full + 8 * s, tile_bytes);
@@ -535,13 +618,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                     if (mine && which >= 2 && which - 2 < Cfg::kHalves)
                         bulk_g2s(sbase + Cfg::kOffV + s * Cfg::kVBytes + (which - 2) * Cfg::kHalfBytes + pg * kPieceBytes,
                                  src + (Cfg::kHalves + which - 2) * kPieceBytes, kPieceBytes, bars + Bars::v_full + 8 * s);
-                    if (!joined) {
-                        __syncthreads();
-                        joined = true;
-                    }
                 }
-                if (!joined) __syncthreads();
-                advance();
+                tile_ctr += n_tiles;
+                ++items_x[0];
+                if (n_x == 2) ++items_x[1];
             }
         } else if (warp == kMmaWarp) {
             // ================================================================
@@ -550,39 +630,62 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
             // descriptors without their start address; a k-step adds its byte offset / 16 to the low word
             const uint64_t desc_kmajor = smem_desc(0, 16, 1024);
             const uint64_t desc_v = smem_desc(0, Cfg::kHalfBytes, 1024);
-            while (next_item()) {
-                __syncthreads();
-                bool ok = true;
-                const int n_x = has_b ? 2 : 1;
-                // S_x(j) = Q_x K(j)^T; the last tile to read K stage s releases it
-                auto issue_qk = [&](int j, int x) {
-                    const uint32_t tc = tile_ctr + j;
-                    const uint32_t s = tc & 1;
-                    if (x == 0) {
-                        ok = wait_all(bars + Bars::k_full + 8 * s, (tc >> 1) & 1, s_abort);
-                        if (!ok) return;
-                        tc_fence_after();
-                    }
-                    if (elect_one()) {
-                        const uint32_t d_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
-                        const uint64_t qd = desc_kmajor + ((sbase + Cfg::kOffQ + x * Cfg::kQBytes) >> 4);
-                        const uint64_t kd = desc_kmajor + ((sbase + Cfg::kOffK + s * Cfg::kKBytes) >> 4);
+            uint32_t n_item = 0, tile_ctr = 0, tiles_x[2] = {0, 0}, items_x[2] = {0, 0};
+            bool ok = true;
+            // S_x = Q_x K^T for key tile number tc (counted over all items) of an item with n_x q tiles.
+            // `first`: the item's first key tile (wait for its Q tile, phase q_par); `last`: its last one
+            // (release the Q buffer).  The last q tile to read K stage s releases it.
+            auto issue_qk = [&](uint32_t tc, int x, int n_x, bool first, bool last, uint32_t q_par) {
+                const uint32_t s = tc & 1;
+                if (x == 0) {
+                    ok = wait_all(bars + Bars::k_full + 8 * s, (tc >> 1) & 1, s_abort);
+                    if (!ok) return;
+                }
+                if (first) {
+                    ok = wait_all(bars + Bars::q_full + 8 * x, q_par & 1, s_abort);
+                    if (!ok) return;
+                }
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint32_t d_addr = tmem + Cfg::kColS + x * Cfg::kColTile;
+                    const uint64_t qd = desc_kmajor + ((sbase + Cfg::kOffQ + x * Cfg::kQBytes) >> 4);
+                    const uint64_t kd = desc_kmajor + ((sbase + Cfg::kOffK + s * Cfg::kKBytes) >> 4);
 #pragma unroll
-                        for (int kk = 0; kk < D / 16; ++kk) {
-                            const uint32_t off = ((kk >> 2) * Cfg::kHalfBytes + (kk & 3) * 32) >> 4;
-                            tc_mma_ss(d_addr, qd + off, kd + off, kIdescQK, kk > 0);
-                        }
-                        tc_commit(bars + Bars::s_full + 8 * x);
-                        if (x == n_x - 1) tc_commit(bars + Bars::k_empty + 8 * s);
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = ((kk >> 2) * Cfg::kHalfBytes + (kk & 3) * 32) >> 4;
+                        tc_mma_ss(d_addr, qd + off, kd + off, kIdescQK, kk > 0);
                     }
-                    __syncwarp();
-                };
-                for (int x = 0; x < n_x && ok; ++x) issue_qk(0, x);
+                    tc_commit(bars + Bars::s_full + 8 * x);
+                    if (x == n_x - 1) tc_commit(bars + Bars::k_empty + 8 * s);
+                    if (last) tc_commit(bars + Bars::q_empty + 8 * x);
+                }
+                __syncwarp();
+            };
+            PrefillItem it, nx;
+            bool have = take_item(n_item, it);
+            ++n_item;
+            bool pre[2] = {false, false};  // S_x of the item's first key tile was issued at the end of the previous item
+            while (have && ok) {
+                const int n_tiles = tiles_of(it);
+                const int n_x = it.n_tok > tile_tok ? 2 : 1;
+                bool have_next = false;
+                int nx_tiles = 0, nx_n_x = 0;
+                for (int x = 0; x < n_x && ok; ++x)
+                    if (!pre[x]) issue_qk(tile_ctr, x, n_x, true, n_tiles == 1, items_x[x]);
+                pre[0] = pre[1] = false;
                 for (int j = 0; j < n_tiles && ok; ++j) {
                     const uint32_t tc = tile_ctr + j;
                     const uint32_t s = tc & 1;
+                    if (j == n_tiles - 1) {
+                        have_next = take_item(n_item, nx);
+                        ++n_item;
+                        if (have_next) {
+                            nx_tiles = tiles_of(nx);
+                            nx_n_x = nx.n_tok > tile_tok ? 2 : 1;
+                        }
+                    }
                     for (int x = 0; x < n_x && ok; ++x) {
-                        ok = wait_all(bars + Bars::p_ready + 8 * x, ((x ? tile_ctr_b : tile_ctr) + j) & 1, s_abort);
+                        ok = wait_all(bars + Bars::p_ready + 8 * x, (tiles_x[x] + j) & 1, s_abort);
                         if (!ok) break;
                         if (x == 0) {
                             ok = wait_all(bars + Bars::v_full + 8 * s, (tc >> 1) & 1, s_abort);
@@ -601,20 +704,29 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                             if (x == n_x - 1) tc_commit(bars + Bars::v_empty + 8 * s);
                         }
                         __syncwarp();
-                        // the tensor pipe runs this thread's MMAs in issue order, so S_x may be
-                        // overwritten by the next QK^T right behind the PV that reads P_x
-                        if (j + 1 < n_tiles) issue_qk(j + 1, x);
+                        // The tensor pipe runs this thread's MMAs in issue order, so S_x may be overwritten by
+                        // the next QK^T right behind the PV that reads P_x -- the next key tile's, or after the
+                        // item's last tile the next item's first (its O_x is not touched before that item's
+                        // first P_x is ready, which the softmax warps signal only after writing this item's
+                        // output).
+                        if (j + 1 < n_tiles) {
+                            issue_qk(tc + 1, x, n_x, false, j + 2 == n_tiles, 0);
+                        } else if (have_next && x < nx_n_x) {
+                            issue_qk(tile_ctr + n_tiles, x, nx_n_x, true, nx_tiles == 1, items_x[x] + 1);
+                            pre[x] = true;
+                        }
                     }
                 }
-                advance();
-            }
-        } else {
-            // the warpgroup's two spare warps only keep the CTA-wide barriers complete
-            while (next_item()) {
-                __syncthreads();
-                advance();
+                tile_ctr += n_tiles;
+                for (int x = 0; x < n_x; ++x) {
+                    tiles_x[x] += n_tiles;
+                    ++items_x[x];
+                }
+                it = nx;
+                have = have_next;
             }
         }
+        // (the warpgroup's two other warps have no work; they wait at the final barrier)
     }
 
     // after an abort: flag the run and give copies in flight a bounded time to land
@@ -623,11 +735,33 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
         for (int s = 0; s < 2; ++s) {
             mbar_wait(bars + Bars::k_full + 8 * s, 0, 200000u);
             mbar_wait(bars + Bars::v_full + 8 * s, 0, 200000u);
+            mbar_wait(bars + Bars::q_full + 8 * s, 0, 200000u);
         }
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
+}
+
+}  // namespace
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up through the runtime so that the library does not link libcuda.
+EncodeTiledFn tensor_map_encoder() {
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return (EncodeTiledFn)f;
+    }();
+    return fn;
 }
 
 }  // namespace
@@ -643,7 +777,6 @@ static ps_status launch_prefill_d(const RunArgs& a) {
     PrefillParams p;
     p.pool = a.pool;
     p.num_pages = a.num_pages;
-    p.q = a.q;
     p.block_table = a.block_table;
     p.max_pages = a.max_pages;
     p.out = a.out;
@@ -658,8 +791,22 @@ static ps_status launch_prefill_d(const RunArgs& a) {
     p.Hkv = a.shape.n_kv_heads;
     p.G = p.Hq / p.Hkv;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+
+    // Q as a [T tokens][Hq heads][D] tensor; a box is one 64-element half of a q tile's 128 rows
+    EncodeTiledFn encode = tensor_map_encoder();
+    if (!encode) return fail(PS_ERR_CUDA, "the driver does not provide cuTensorMapEncodeTiled");
+    CUtensorMap q_map;
+    const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)p.Hq, (cuuint64_t)a.total_q};
+    const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)p.Hq * D * 2};
+    const cuuint32_t box[3] = {64, (cuuint32_t)p.G, (cuuint32_t)(kRows / p.G)};
+    const cuuint32_t elem_strides[3] = {1, 1, 1};
+    const CUresult r = encode(&q_map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<__nv_bfloat16*>(a.q), dims, strides, box,
+                              elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(PS_ERR_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+
     const int grid = a.w.n_prefill_ctas > 0 ? a.w.n_prefill_ctas : (a.w.n_prefill < a.pf_sms ? a.w.n_prefill : a.pf_sms);
-    prefill_kernel<D><<<grid, kThreads, Cfg::kSmemBytes, a.stream>>>(p);
+    prefill_kernel<D><<<grid, kThreads, Cfg::kSmemBytes, a.stream>>>(p, q_map);
     PS_CUDA_TRY(cudaGetLastError());
     return PS_OK;
 }
