@@ -22,7 +22,8 @@ constexpr int kPrefillKeyTile = 128;    // keys per tensor-core tile
 // Measured on B200 (decode: bandwidth against the number of SMs the kernel runs on; prefill: time of one
 // key-tile step of a q tile pair), used to split the SMs of a mixed batch between the two kernels.
 constexpr double kDecodePeakBytesPerSec = 6.7e12;
-constexpr double kDecodeBytesPerSecPerSm = 125e9;
+constexpr double kDecodeSharedPeakBytesPerSec = 6.0e12;  // decode rows beside a running prefill kernel
+constexpr double kDecodeBytesPerSecPerSm = 115e9;
 constexpr double kPrefillStepSec = 2.5e-6;
 constexpr double kKernelFloorSec = 12e-6;
 
@@ -339,18 +340,25 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
         pl->dec_sms = pl->pf_sms = pl->num_sms;
         pl->concurrent = false;
         if (dec_bytes > 0 && pf_steps > 0 && pl->num_sms >= 16) {
-            // time models (seconds): decode = bytes / min(peak, n * per-SM rate); prefill = steps * step time / m
+            // time models (seconds): decode = bytes / min(side-by-side peak, n * per-SM rate); prefill = steps * step time / m
+            auto t_dec = [&](int nd) { return dec_bytes / std::min(kDecodeSharedPeakBytesPerSec, nd * kDecodeBytesPerSecPerSm) + kKernelFloorSec; };
+            auto t_pf = [&](int nd) { return pf_steps * kPrefillStepSec / (pl->num_sms - nd) + kKernelFloorSec; };
             int best_n = 0;
             double best_t = 1e30;
             for (int nd = 8; nd <= pl->num_sms - 8; nd += 4) {
-                const double t_dec = dec_bytes / std::min(kDecodePeakBytesPerSec, nd * kDecodeBytesPerSecPerSm) + kKernelFloorSec;
-                const double t_pf = pf_steps * kPrefillStepSec / (pl->num_sms - nd) + kKernelFloorSec;
-                const double t = std::max(t_dec, t_pf);
+                const double t = std::max(t_dec(nd), t_pf(nd));
                 if (t < best_t) {
                     best_t = t;
                     best_n = nd;
                 }
             }
+            // Once the decode rows saturate HBM the modelled time is flat in n; measured step times keep
+            // improving a little as the decode kernel gets more SMs, as long as the prefill kernel still ends
+            // well before it.  Take the middle of that flat stretch.
+            int hi = best_n;
+            for (int nd = best_n; nd <= pl->num_sms - 8; nd += 4)
+                if (std::max(t_dec(nd), t_pf(nd)) <= 1.015 * best_t && t_pf(nd) <= 0.8 * t_dec(nd)) hi = nd;
+            best_n = (best_n + hi) / 2 / 4 * 4;
             const double t_seq = dec_bytes / kDecodePeakBytesPerSec + pf_steps * kPrefillStepSec / pl->num_sms + 2 * kKernelFloorSec;
             if (best_n > 0 && best_t < 0.95 * t_seq) {
                 pl->dec_sms = best_n;
