@@ -143,8 +143,10 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
 }
 
 // Cost model of the prefill kernel in units of one 128-key tile step: an item pays a fixed
-// overhead (Q load, pipeline fill, epilogue) plus one unit per key tile.
-constexpr double kPrefillFixedCost = 2.0;
+// overhead (pipeline fill, output) plus one unit per key tile.
+// (fitted to per-CTA run times on B200: 2.2 us per step, about 3 us per item, 1.2 us more for a masked tile)
+constexpr double kPrefillFixedCost = 1.5;
+constexpr double kPrefillMaskedExtra = 0.5;  // the diagonal tile of an item takes the slower masked softmax
 constexpr double kPrefillMinCtaCost = 4.0;  // do not spread the work thinner than this per CTA (two key tiles)
 
 static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len, const std::vector<int32_t>& q_start,
@@ -189,37 +191,53 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
         // line, cutting items where a share ends.  Only the cut items need the merge.
         static_partition = true;
         double total = 0;
-        for (const Tile& t : tiles) total += kPrefillFixedCost + t.key_tiles;
+        for (const Tile& t : tiles) total += kPrefillFixedCost + t.key_tiles + kPrefillMaskedExtra;
         const int n_cta = (int)std::max<double>(1, std::min<double>(pl->pf_sms, total / kPrefillMinCtaCost));
-        const double quota = total / n_cta;
-        pl->prefill_cta_start.assign(1, 0);
-        double cum = 0, boundary = quota;
-        int n_items = 0, cta = 0;
-        for (size_t i = 0; i < tiles.size(); ++i) {
-            const int kt = tiles[i].key_tiles;
-            const double tile_end = cum + kPrefillFixedCost + kt;
-            int kt0 = 0;
-            while (cta < n_cta - 1 && boundary < tile_end - 0.5) {
-                int cut = (int)std::lround(boundary - cum - kPrefillFixedCost);
-                cut = std::max(cut, kt0);
-                if (cut >= kt) break;
-                if (cut > kt0) {
-                    cuts[i].push_back(cut);
-                    kt0 = cut;
-                    ++n_items;
+        // CTA k ends where the running cost passes (k + 1) * quota (absolute marks, so rounding does not pile
+        // up).  A share that ends inside an item makes the rest of that item pay the fixed cost again, and how
+        // many shares do depends on the quota itself: bisect for the smallest quota that does not leave the
+        // last CTA with more than a share.
+        int n_items = 0;
+        double q_lo = total / n_cta, q_hi = (total + (n_cta - 1) * kPrefillFixedCost) / n_cta + 0.5;
+        for (int pass = 0; pass < 7; ++pass) {
+            const double quota = pass == 6 ? q_hi : 0.5 * (q_lo + q_hi);  // the last pass keeps a quota known to fit
+            pl->prefill_cta_start.assign(1, 0);
+            for (auto& c : cuts) c.clear();
+            n_items = 0;
+            int cta = 0;
+            double cum = 0, cum_at_last = 0;  // cost handed out so far; and before the last CTA
+            auto close_cta = [&]() {
+                ++cta;
+                pl->prefill_cta_start.push_back(n_items);
+                if (cta == n_cta - 1) cum_at_last = cum;
+            };
+            for (size_t i = 0; i < tiles.size(); ++i) {
+                const int kt = tiles[i].key_tiles;
+                int kt0 = 0;
+                for (;;) {
+                    const double rest = kPrefillFixedCost + (kt - kt0) + kPrefillMaskedExtra;  // the item's remaining tiles as one piece
+                    const double room = (cta + 1) * quota - cum;
+                    const bool cta_has_work = pl->prefill_cta_start.back() < n_items;
+                    const int take = (int)std::lround(room - kPrefillFixedCost);
+                    if (cta == n_cta - 1 || rest <= room + 0.5 || take >= kt - kt0 || (take < 1 && !cta_has_work)) {
+                        cum += rest;
+                        ++n_items;
+                        break;
+                    }
+                    if (take >= 1) {
+                        kt0 += take;
+                        cuts[i].push_back(kt0);
+                        cum += kPrefillFixedCost + take;
+                        ++n_items;
+                    }
+                    close_cta();  // (with take < 1: no room left for even one key tile; the item starts in the next CTA)
                 }
-                ++cta;
-                pl->prefill_cta_start.push_back(n_items);
-                boundary += quota;
+                while (cta < n_cta - 1 && cum >= (cta + 1) * quota - 0.5) close_cta();
             }
-            ++n_items;
-            cum = tile_end;
-            while (cta < n_cta - 1 && boundary <= cum + 0.5) {
-                ++cta;
-                pl->prefill_cta_start.push_back(n_items);
-                boundary += quota;
-            }
+            const bool fits = cta < n_cta - 1 || cum - cum_at_last <= quota + 0.5;
+            if (fits) q_hi = quota; else q_lo = quota;
         }
+        while ((int)pl->prefill_cta_start.size() < n_cta) pl->prefill_cta_start.push_back(n_items);  // CTAs left without work
         pl->prefill_cta_start.push_back(n_items);
     }
 
