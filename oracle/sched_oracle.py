@@ -1,0 +1,139 @@
+"""CPU oracle for the scheduler-side consumers of the latency table (test infrastructure).
+
+Plain, slow Python written from the paper's text; only the tests and the
+bench scripts' baseline legs may import it, the library and its binding never
+do.  Every function simulates or enumerates directly -- no sweeps, no sorting
+tricks, no closed forms -- so that it can be checked against the paper by eye.
+
+Notation (paper section 4.5): a running decode request holds ``kv_len`` tokens
+in the cache (the token of the coming iteration included) and still has
+``remaining`` tokens to generate (that one included).  Iterations are numbered
+t = 0, 1, ... from the coming one; the request takes part in iterations
+0 .. remaining - 1 and holds ``kv_len + t`` tokens in iteration t.
+
+parity pins: tests/test_sched_oracle_pins.py (the paper's chunk-schedule
+example, closed forms, numpy's least-squares routine, brute force by explicit
+matrices).
+"""
+from __future__ import annotations
+
+
+# ---------------------------------------------------------------------------
+# latency table (section 4.5: a profiled map of (batch size, KV cache size) to execution time)
+# ---------------------------------------------------------------------------
+def table_build(rows):
+    """rows: iterable of (token_batch, kv_tokens, latency_us).  Returns the table as a list of lines
+    (token_batch, intercept_us, slope_us_per_token) sorted by token_batch: per batch size the ordinary
+    least-squares straight line of latency over KV tokens (iteration time is affine in the KV-cache
+    size at a fixed batch size, section 3.4)."""
+    groups = {}
+    for b, kv, lat in rows:
+        groups.setdefault(int(b), []).append((float(kv), float(lat)))
+    lines = []
+    for b in sorted(groups):
+        pts = groups[b]
+        n = len(pts)
+        mean_x = sum(x for x, _ in pts) / n
+        mean_y = sum(y for _, y in pts) / n
+        sxx = sum((x - mean_x) * (x - mean_x) for x, _ in pts)
+        sxy = sum((x - mean_x) * (y - mean_y) for x, y in pts)
+        slope = sxy / sxx if sxx > 0.0 else 0.0
+        lines.append((b, mean_y - slope * mean_x, slope))
+    return lines
+
+
+def table_predict(lines, token_batch, kv_tokens):
+    """Predicted iteration time: the line of that batch size evaluated at kv_tokens; between two lines their
+    two values interpolated linearly in the batch size; outside the lines the nearest line as it is."""
+    lines = sorted(lines)
+    at = lambda ln: ln[1] + ln[2] * float(kv_tokens)
+    if token_batch <= lines[0][0]:
+        return at(lines[0])
+    if token_batch >= lines[-1][0]:
+        return at(lines[-1])
+    for lo, hi in zip(lines[:-1], lines[1:]):
+        if lo[0] <= token_batch < hi[0]:
+            w = (token_batch - lo[0]) / float(hi[0] - lo[0])
+            return at(lo) + (at(hi) - at(lo)) * w
+    raise AssertionError("unreachable")
+
+
+# ---------------------------------------------------------------------------
+# decode admission (section 4.5: simulate future iterations, take the largest KV-cache size)
+# ---------------------------------------------------------------------------
+def kv_at(kv_len, remaining, t):
+    """Total KV tokens and number of requests in iteration t."""
+    alive = [L + t for L, R in zip(kv_len, remaining) if R > t]
+    return sum(alive), len(alive)
+
+
+def peak_kv(kv_len, remaining):
+    """(largest total KV-cache size over the future iterations, first iteration where it occurs)."""
+    peak, when = 0, 0
+    horizon = max(remaining) if len(remaining) else 0
+    for t in range(horizon):  # "simulates future iterations ... and exits when finished"
+        kv, _ = kv_at(kv_len, remaining, t)
+        if kv > peak:
+            peak, when = kv, t
+    return peak, when
+
+
+def admit(lines, kv_len, remaining, new_kv_len, new_remaining, extra_tokens, tpot_us):
+    """(admitted?, predicted iteration time, peak KV) for one new decode request: the table at the current
+    token batch size and the largest future KV-cache size must stay below the TPOT."""
+    peak, _ = peak_kv(list(kv_len) + [new_kv_len], list(remaining) + [new_remaining])
+    batch = len(kv_len) + 1 + extra_tokens
+    pred = table_predict(lines, batch, peak)
+    return pred < tpot_us, pred, peak
+
+
+# ---------------------------------------------------------------------------
+# prefill chunking (section 4.7)
+# ---------------------------------------------------------------------------
+def chunk_next(remaining, budget, used, dynamic):
+    """Chunk length per request for the coming iteration, first come first served.  Dynamic chunking: a request
+    with fewer than two budgets of prompt left is finished at once and nobody is admitted behind it."""
+    left = budget - used
+    out = [0] * len(remaining)
+    for i, rem in enumerate(remaining):
+        if left <= 0:
+            break
+        if dynamic and rem < 2 * budget:
+            out[i] = rem
+            break
+        out[i] = min(rem, left)
+        left -= out[i]
+    return out
+
+
+def chunk_schedule(prompt_len, budget, first_free, dynamic):
+    """All chunks of one prompt; the first iteration has only first_free tokens of its budget left."""
+    chunks, rem, used = [], prompt_len, budget - first_free
+    while rem > 0:
+        c = chunk_next([rem], budget, used, dynamic)[0]
+        if c > 0:
+            chunks.append(c)
+            rem -= c
+        used = 0
+    return chunks
+
+
+def chunk_predict(lines, kv_len, remaining, prompt_len, max_chunk, tpot_us):
+    """Continuous chunked-prefill prediction.  Returns (chunk, iterations, completion_us, maintained)."""
+    kv0, n0 = kv_at(kv_len, remaining, 0)
+    chunk = 0
+    for c in range(min(prompt_len, max_chunk), 0, -1):
+        if table_predict(lines, n0 + c, kv0 + c) <= tpot_us:
+            chunk = c
+            break
+    if chunk == 0:
+        return 0, 0, 0.0, False
+    iters = -(-prompt_len // chunk)  # ceil
+    completion, maintained = 0.0, True
+    for k in range(iters):
+        kv, n = kv_at(kv_len, remaining, k)
+        c_k = min(chunk, prompt_len - k * chunk)
+        pred = table_predict(lines, n + c_k, kv + min((k + 1) * chunk, prompt_len))
+        completion += pred
+        maintained = maintained and pred <= tpot_us
+    return chunk, iters, completion, maintained

@@ -1,0 +1,183 @@
+"""Pins of the scheduler-side oracle (oracle/sched_oracle.py) against things other than itself: the paper's
+worked chunk-schedule example (section 4.7), closed forms, numpy's least-squares routine and explicit-matrix
+brute force."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import sched_oracle as so
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def read_example():
+    out = {}
+    for line in open(os.path.join(HERE, "golden", "dynamic_chunking_example.txt")):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            name, *vals = line.split()
+            out[name] = [int(v) for v in vals]
+    return out
+
+
+# ---------------------------------------------------------------------------
+# chunk schedules: the paper's example, section 4.7
+# ---------------------------------------------------------------------------
+def test_chunk_schedules_of_the_papers_example():
+    ex = read_example()
+    budget, prompt = ex["budget"][0], ex["prompt"][0]
+    assert so.chunk_schedule(prompt, budget, budget, dynamic=False) == ex["static"]
+    assert so.chunk_schedule(prompt, budget, 1, dynamic=False) == ex["static_worst"]
+    assert so.chunk_schedule(prompt, budget, budget, dynamic=True) == ex["dynamic"]
+    # "allows almost every request to reduce one iteration": the worst case drops from four iterations to three
+    worst_dynamic = so.chunk_schedule(prompt, budget, 1, dynamic=True)
+    assert worst_dynamic == [1, 1024, 1025] and len(worst_dynamic) == len(ex["static_worst"]) - 1
+
+
+def test_chunk_schedule_invariants():
+    rng = np.random.default_rng(5)
+    for _ in range(300):
+        budget = int(rng.integers(1, 600))
+        prompt = int(rng.integers(1, 6 * budget + 2))
+        free = int(rng.integers(1, budget + 1))
+        st = so.chunk_schedule(prompt, budget, free, False)
+        dy = so.chunk_schedule(prompt, budget, free, True)
+        assert sum(st) == prompt and sum(dy) == prompt
+        assert st[0] <= free and all(c <= budget for c in st)
+        # static chunking is ceil((prompt - first) / budget) + 1 iterations
+        first = min(prompt, free)
+        assert len(st) == 1 + -(-(prompt - first) // budget)
+        assert all(c < 2 * budget for c in dy) and len(dy) <= len(st)
+        # only the last dynamic chunk may exceed what was free in its iteration
+        assert all(c <= budget for c in dy[:-1])
+
+
+def test_chunk_next_is_first_come_first_served():
+    # plain chunked prefill fills the budget in order
+    assert so.chunk_next([300, 500, 900], 1024, 0, False) == [300, 500, 224]
+    assert so.chunk_next([300, 500, 900], 1024, 1000, False) == [24, 0, 0]
+    assert so.chunk_next([300], 1024, 1024, False) == [0]
+    # dynamic: the first request with fewer than two budgets left is finished at once and closes the iteration
+    assert so.chunk_next([5000, 1500, 10], 1024, 0, True) == [1024, 0, 0]
+    assert so.chunk_next([2047, 10], 1024, 0, True) == [2047, 0]
+    assert so.chunk_next([2048, 10], 1024, 0, True) == [1024, 0]
+    assert so.chunk_next([3000, 10], 1024, 1000, True) == [24, 0]
+    assert so.chunk_next([10, 3000], 1024, 1000, True) == [10, 0]
+
+
+# ---------------------------------------------------------------------------
+# peak KV of the simulated future iterations, section 4.5
+# ---------------------------------------------------------------------------
+def test_peak_kv_closed_forms():
+    # one request: it grows by one token per iteration until its last one
+    assert so.peak_kv([100], [7]) == (106, 6)
+    # equal remaining lengths: everybody is there until the end
+    assert so.peak_kv([10, 20, 30], [5, 5, 5]) == (60 + 3 * 4, 4)
+    # a long context that leaves at once dominates: the peak is now
+    assert so.peak_kv([10, 1000], [3, 1]) == (1010, 0)
+    # worked by hand: t0 = 5+6+7 = 18, t1 = 6+7 = 13 (third left), t2 = 7 (second left)
+    assert so.peak_kv([5, 6, 7], [3, 2, 1]) == (18, 0)
+    assert so.peak_kv([5, 6, 7], [4, 4, 1]) == (18, 0)   # t0 18, t1 13, t2 15, t3 17
+    assert so.peak_kv([5, 6, 7], [5, 5, 1]) == (19, 4)   # ... t4 = 9 + 10 = 19
+    assert so.peak_kv([10, 3], [4, 1]) == (13, 0)        # t0 13, t1 11, t2 12, t3 13: a tie reports the first
+    assert so.peak_kv([], []) == (0, 0)
+
+
+def test_peak_kv_against_explicit_matrix():
+    rng = np.random.default_rng(11)
+    for _ in range(200):
+        n = int(rng.integers(1, 40))
+        kv = rng.integers(1, 5000, n)
+        rem = rng.integers(1, 300, n)
+        t = np.arange(rem.max())[:, None]                       # iterations x requests
+        total = ((kv[None, :] + t) * (rem[None, :] > t)).sum(axis=1)
+        assert so.peak_kv(kv.tolist(), rem.tolist()) == (int(total.max()), int(total.argmax()))
+
+
+def test_peak_kv_monotone_in_the_request_set():
+    rng = np.random.default_rng(12)
+    for _ in range(100):
+        n = int(rng.integers(1, 20))
+        kv, rem = rng.integers(1, 3000, n).tolist(), rng.integers(1, 200, n).tolist()
+        base, _ = so.peak_kv(kv, rem)
+        more, _ = so.peak_kv(kv + [int(rng.integers(1, 3000))], rem + [int(rng.integers(1, 200))])
+        assert more > base  # the newcomer is present at iteration 0 at least... and at the old peak or earlier
+        assert more >= so.kv_at(kv, rem, 0)[0]
+
+
+# ---------------------------------------------------------------------------
+# table: least-squares lines and the lookup
+# ---------------------------------------------------------------------------
+def test_table_fit_recovers_exact_lines_and_matches_numpy():
+    rng = np.random.default_rng(3)
+    rows = []
+    truth = {72: (15.0, 2.5e-4), 320: (40.0, 3.0e-4), 2304: (310.0, 1.0e-4)}
+    for b, (a, s) in truth.items():
+        for kv in rng.integers(1000, 2_000_000, 27):
+            rows.append((b, int(kv), a + s * float(kv)))
+    lines = so.table_build(rows)
+    assert [ln[0] for ln in lines] == sorted(truth)
+    for b, a, s in lines:
+        assert abs(a - truth[b][0]) < 1e-6 and abs(s - truth[b][1]) < 1e-12
+    # noisy data: the same coefficients as numpy's least squares
+    noisy = [(b, kv, lat * (1.0 + 0.05 * rng.standard_normal())) for b, kv, lat in rows]
+    for b, a, s in so.table_build(noisy):
+        x = np.array([kv for bb, kv, _ in noisy if bb == b], dtype=np.float64)
+        y = np.array([lat for bb, _, lat in noisy if bb == b], dtype=np.float64)
+        coef, *_ = np.linalg.lstsq(np.stack([np.ones_like(x), x], axis=1), y, rcond=None)
+        assert abs(a - coef[0]) < 1e-6 * max(1.0, abs(coef[0])) and abs(s - coef[1]) < 1e-9 * abs(coef[1])
+    # a line whose rows share one KV size: slope 0 and their mean
+    flat = so.table_build([(8, 500, 10.0), (8, 500, 14.0)])
+    assert flat == [(8, 12.0, 0.0)]
+
+
+def test_table_lookup_interpolates_in_batch_and_clamps():
+    lines = [(100, 10.0, 1e-3), (300, 50.0, 2e-3)]
+    assert so.table_predict(lines, 100, 1000) == pytest.approx(11.0)
+    assert so.table_predict(lines, 300, 1000) == pytest.approx(52.0)
+    assert so.table_predict(lines, 200, 1000) == pytest.approx(0.5 * (11.0 + 52.0))   # midpoint
+    assert so.table_predict(lines, 150, 0) == pytest.approx(10.0 + 0.25 * 40.0)
+    assert so.table_predict(lines, 5, 1000) == pytest.approx(11.0)                   # below: first line
+    assert so.table_predict(lines, 9000, 1000) == pytest.approx(52.0)                # above: last line
+    assert so.table_predict(list(reversed(lines)), 200, 1000) == pytest.approx(31.5)  # order of the lines is free
+
+
+def test_admission_uses_the_peak_and_the_current_batch_size():
+    # table(b, kv) = 2 b + 0.01 kv
+    lines = [(1, 2.0, 0.01), (1001, 2002.0, 0.01)]
+    kv, rem = [100, 200], [10, 3]
+    # with the newcomer (50 tokens, 5 to go): t0 = 350, t1 = 353, t2 = 356, t3 = 103+53 = 156, t4 = 158 -> peak 356
+    ok, pred, peak = so.admit(lines, kv, rem, 50, 5, 0, 10.0)
+    assert peak == 356 and pred == pytest.approx(2 * 3 + 3.56) and ok
+    assert not so.admit(lines, kv, rem, 50, 5, 0, 9.56)[0]          # strictly below the TPOT is required
+    assert so.admit(lines, kv, rem, 50, 5, 0, 9.5601)[0]
+    # prefill tokens batched alongside count in the batch size only
+    ok, pred, peak = so.admit(lines, kv, rem, 50, 5, 100, 1e9)
+    assert peak == 356 and pred == pytest.approx(2 * 103 + 3.56)
+
+
+def test_chunk_prediction_closed_form():
+    # table(b, kv) = alpha b + beta kv, no decode requests: chunk c costs (alpha + beta) c in iteration 0
+    alpha, beta = 0.1, 0.002
+    lines = [(1, alpha, beta), (100001, alpha * 100001, beta)]
+    tpot = 50.0
+    c, iters, total, kept = so.chunk_predict(lines, [], [], 3000, 2048, tpot)
+    assert c == int(tpot / (alpha + beta))                       # 490
+    assert iters == -(-3000 // c)
+    # iteration k costs alpha c_k + beta min((k + 1) c, P); it grows with k, so the chunk size is not kept
+    want = sum(alpha * min(c, 3000 - k * c) + beta * min((k + 1) * c, 3000) for k in range(iters))
+    assert total == pytest.approx(want) and not kept
+    # with beta = 0 the cost does not grow: the chunk is kept
+    lines0 = [(1, alpha, 0.0), (100001, alpha * 100001, 0.0)]
+    c, iters, total, kept = so.chunk_predict(lines0, [], [], 3000, 2048, tpot)
+    assert c == 500 and iters == 6 and kept and total == pytest.approx(alpha * 3000)
+    # decode requests take their share: alpha (n + c) + beta (KV + c) <= tpot
+    kv, rem = [1000] * 20, [1000] * 20
+    c, *_ = so.chunk_predict(lines, kv, rem, 3000, 2048, tpot)
+    assert c == int((tpot - alpha * 20 - beta * 20000) / (alpha + beta) + 1e-9)
+    # no chunk fits
+    assert so.chunk_predict(lines, [10 ** 6], [5], 100, 2048, tpot) == (0, 0, 0.0, False)
+    # the cap and the prompt length bound the chunk
+    assert so.chunk_predict(lines0, [], [], 3000, 128, tpot)[0] == 128
+    assert so.chunk_predict(lines0, [], [], 77, 2048, tpot)[:2] == (77, 1)
