@@ -35,7 +35,7 @@ def sources():
 
 
 def _deps_mtime() -> float:
-    files = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + [os.path.join(HERE, "..", "include", "polyserve_attn.h")]
+    files = sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(HERE, "..", "include", "*.h"))
     return max(os.path.getmtime(f) for f in files)
 
 

@@ -1,0 +1,290 @@
+// Host-side consumers of the profiled latency table: the table itself, the
+// decode admission test (paper section 4.5) and the prefill chunk sizers
+// (section 4.7).  Plain host code; nothing here touches the device.
+#include <algorithm>
+#include <cmath>
+#include <new>
+#include <numeric>
+#include <vector>
+
+#include "common.cuh"
+#include "../../include/polyserve_sched.h"
+
+struct ps_table {
+    std::vector<int32_t> batch;   // sorted, distinct
+    std::vector<double> intercept;
+    std::vector<double> slope;
+};
+
+namespace ps {
+namespace {
+
+double line_at(const ps_table& t, size_t i, int64_t kv) { return t.intercept[i] + t.slope[i] * (double)kv; }
+
+double predict(const ps_table& t, int32_t token_batch, int64_t kv) {
+    const size_t n = t.batch.size();
+    if (token_batch <= t.batch.front()) return line_at(t, 0, kv);
+    if (token_batch >= t.batch.back()) return line_at(t, n - 1, kv);
+    // lines lo, hi with batch[lo] <= token_batch < batch[hi]
+    const size_t hi = (size_t)(std::upper_bound(t.batch.begin(), t.batch.end(), token_batch) - t.batch.begin());
+    const size_t lo = hi - 1;
+    const double w = (double)(token_batch - t.batch[lo]) / (double)(t.batch[hi] - t.batch[lo]);
+    const double a = line_at(t, lo, kv), b = line_at(t, hi, kv);
+    return a + (b - a) * w;
+}
+
+ps_status check_requests(const int32_t* kv_len, const int32_t* remaining, int32_t n) {
+    if (n < 0 || (n > 0 && (!kv_len || !remaining))) return fail(PS_ERR_INVALID, "request arrays: n = %d with a null pointer", n);
+    for (int32_t i = 0; i < n; ++i)
+        if (kv_len[i] < 1 || remaining[i] < 1)
+            return fail(PS_ERR_INVALID, "request %d: kv_len = %d, remaining = %d (both must be >= 1)", i, kv_len[i], remaining[i]);
+    return PS_OK;
+}
+
+// The decode requests of an instance ordered by the iteration at which they leave, with running sums, so
+// that the requests alive in iteration t (remaining > t) and their total length are a suffix.
+struct Future {
+    std::vector<int32_t> rem;      // ascending
+    std::vector<int64_t> len_suf;  // len_suf[i] = sum of kv_len over sorted positions >= i (n + 1 entries)
+    Future(const int32_t* kv_len, const int32_t* remaining, int32_t n) : rem(n), len_suf(n + 1, 0) {
+        std::vector<int32_t> order(n);
+        std::iota(order.begin(), order.end(), 0);
+        std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return remaining[a] < remaining[b]; });
+        for (int32_t i = 0; i < n; ++i) rem[i] = remaining[order[i]];
+        for (int32_t i = n - 1; i >= 0; --i) len_suf[i] = len_suf[i + 1] + kv_len[order[i]];
+    }
+    // first sorted position alive in iteration t; `from` is a position known not to be past it
+    size_t first_alive(int64_t t, size_t from = 0) const {
+        while (from < rem.size() && rem[from] <= t) ++from;
+        return from;
+    }
+    int64_t kv(size_t pos, int64_t t) const { return len_suf[pos] + (int64_t)(rem.size() - pos) * t; }
+    // Between two departures the total grows by one token per request and iteration, so the largest
+    // value before each departure is in the last iteration of the requests that leave.
+    void peak(int64_t* peak_out, int32_t* iter_out) const {
+        int64_t best = 0;
+        int32_t when = 0;
+        for (size_t i = 0; i < rem.size(); ++i) {
+            if (i > 0 && rem[i] == rem[i - 1]) continue;
+            const int64_t t = (int64_t)rem[i] - 1;
+            const int64_t v = kv(i, t);
+            if (v > best) best = v, when = (int32_t)t;
+        }
+        *peak_out = best;
+        *iter_out = when;
+    }
+};
+
+}  // namespace
+}  // namespace ps
+
+using ps::fail;
+
+extern "C" {
+
+ps_status ps_table_from_lines(const int32_t* token_batch, const double* intercept_us, const double* slope_us_per_token,
+                              int32_t n_lines, ps_table** out) {
+    ps::clear_error();
+    if (!token_batch || !intercept_us || !slope_us_per_token || !out || n_lines < 1)
+        return fail(PS_ERR_INVALID, "ps_table_from_lines: null pointer or n_lines < 1");
+    std::vector<int32_t> order(n_lines);
+    std::iota(order.begin(), order.end(), 0);
+    std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return token_batch[a] < token_batch[b]; });
+    ps_table* t = new (std::nothrow) ps_table;
+    if (!t) return fail(PS_ERR_OOM, "ps_table_from_lines: out of host memory");
+    for (int32_t k = 0; k < n_lines; ++k) {
+        const int32_t i = order[k];
+        if (token_batch[i] < 1 || !std::isfinite(intercept_us[i]) || !std::isfinite(slope_us_per_token[i]) ||
+            (k > 0 && token_batch[i] == token_batch[order[k - 1]])) {
+            delete t;
+            return fail(PS_ERR_INVALID, "ps_table_from_lines: line %d (token_batch %d) is not usable or is a duplicate", i, token_batch[i]);
+        }
+        t->batch.push_back(token_batch[i]);
+        t->intercept.push_back(intercept_us[i]);
+        t->slope.push_back(slope_us_per_token[i]);
+    }
+    *out = t;
+    return PS_OK;
+}
+
+ps_status ps_table_build(const ps_grid_row* rows, int64_t n_rows, ps_table** out) {
+    ps::clear_error();
+    if (!rows || !out || n_rows < 1) return fail(PS_ERR_INVALID, "ps_table_build: null pointer or n_rows < 1");
+    for (int64_t i = 0; i < n_rows; ++i)
+        if (rows[i].token_batch < 1 || rows[i].kv_tokens < 0 || !std::isfinite(rows[i].latency_us))
+            return fail(PS_ERR_INVALID, "ps_table_build: row %lld has token_batch %d, kv_tokens %lld, latency %g", (long long)i,
+                        rows[i].token_batch, (long long)rows[i].kv_tokens, (double)rows[i].latency_us);
+    // rows of one batch size together, in their input order
+    std::vector<int64_t> order(n_rows);
+    std::iota(order.begin(), order.end(), (int64_t)0);
+    std::stable_sort(order.begin(), order.end(), [&](int64_t a, int64_t b) { return rows[a].token_batch < rows[b].token_batch; });
+    std::vector<int32_t> batch;
+    std::vector<double> icpt, slope;
+    for (int64_t g0 = 0; g0 < n_rows;) {
+        int64_t g1 = g0;
+        while (g1 < n_rows && rows[order[g1]].token_batch == rows[order[g0]].token_batch) ++g1;
+        const double n = (double)(g1 - g0);
+        double sum_x = 0.0, sum_y = 0.0;
+        for (int64_t k = g0; k < g1; ++k) sum_x += (double)rows[order[k]].kv_tokens, sum_y += (double)rows[order[k]].latency_us;
+        const double mean_x = sum_x / n, mean_y = sum_y / n;
+        double sxx = 0.0, sxy = 0.0;
+        for (int64_t k = g0; k < g1; ++k) {
+            const double dx = (double)rows[order[k]].kv_tokens - mean_x;
+            sxx += dx * dx;
+            sxy += dx * ((double)rows[order[k]].latency_us - mean_y);
+        }
+        const double s = sxx > 0.0 ? sxy / sxx : 0.0;
+        batch.push_back(rows[order[g0]].token_batch);
+        slope.push_back(s);
+        icpt.push_back(mean_y - s * mean_x);
+        g0 = g1;
+    }
+    return ps_table_from_lines(batch.data(), icpt.data(), slope.data(), (int32_t)batch.size(), out);
+}
+
+ps_status ps_table_free(ps_table* table) {
+    delete table;
+    return PS_OK;
+}
+
+ps_status ps_table_size(const ps_table* table, int32_t* n_lines_out) {
+    ps::clear_error();
+    if (!table || !n_lines_out) return fail(PS_ERR_INVALID, "ps_table_size: null pointer");
+    *n_lines_out = (int32_t)table->batch.size();
+    return PS_OK;
+}
+
+ps_status ps_table_get_lines(const ps_table* table, int32_t* token_batch_out, double* intercept_us_out,
+                             double* slope_us_per_token_out, int32_t capacity) {
+    ps::clear_error();
+    if (!table) return fail(PS_ERR_INVALID, "ps_table_get_lines: null table");
+    if (capacity < (int32_t)table->batch.size()) return fail(PS_ERR_INVALID, "ps_table_get_lines: capacity %d < %zu lines", capacity, table->batch.size());
+    for (size_t i = 0; i < table->batch.size(); ++i) {
+        if (token_batch_out) token_batch_out[i] = table->batch[i];
+        if (intercept_us_out) intercept_us_out[i] = table->intercept[i];
+        if (slope_us_per_token_out) slope_us_per_token_out[i] = table->slope[i];
+    }
+    return PS_OK;
+}
+
+ps_status ps_table_predict(const ps_table* table, int32_t token_batch, int64_t kv_tokens, double* latency_us_out) {
+    ps::clear_error();
+    if (!table || !latency_us_out) return fail(PS_ERR_INVALID, "ps_table_predict: null pointer");
+    if (token_batch < 1 || kv_tokens < 0) return fail(PS_ERR_INVALID, "ps_table_predict: token_batch %d, kv_tokens %lld", token_batch, (long long)kv_tokens);
+    *latency_us_out = ps::predict(*table, token_batch, kv_tokens);
+    return PS_OK;
+}
+
+ps_status ps_peak_kv(const int32_t* kv_len, const int32_t* remaining, int32_t n, int64_t* peak_kv_out, int32_t* peak_iter_out) {
+    ps::clear_error();
+    if (!peak_kv_out || !peak_iter_out) return fail(PS_ERR_INVALID, "ps_peak_kv: null output");
+    if (ps_status st = ps::check_requests(kv_len, remaining, n)) return st;
+    ps::Future(kv_len, remaining, n).peak(peak_kv_out, peak_iter_out);
+    return PS_OK;
+}
+
+ps_status ps_admit(const ps_table* table, const int32_t* kv_len, const int32_t* remaining, int32_t n_running, int32_t new_kv_len,
+                   int32_t new_remaining, int32_t extra_tokens, double tpot_us, int32_t* admit_out, double* predicted_us_out,
+                   int64_t* peak_kv_out) {
+    ps::clear_error();
+    if (!table) return fail(PS_ERR_INVALID, "ps_admit: null table");
+    if (extra_tokens < 0) return fail(PS_ERR_INVALID, "ps_admit: extra_tokens %d < 0", extra_tokens);
+    if (ps_status st = ps::check_requests(kv_len, remaining, n_running)) return st;
+    if (ps_status st = ps::check_requests(&new_kv_len, &new_remaining, 1)) return st;
+    std::vector<int32_t> len(kv_len, kv_len + n_running), rem(remaining, remaining + n_running);
+    len.push_back(new_kv_len);
+    rem.push_back(new_remaining);
+    int64_t peak = 0;
+    int32_t when = 0;
+    ps::Future(len.data(), rem.data(), n_running + 1).peak(&peak, &when);
+    const double pred = ps::predict(*table, n_running + 1 + extra_tokens, peak);
+    if (admit_out) *admit_out = pred < tpot_us ? 1 : 0;
+    if (predicted_us_out) *predicted_us_out = pred;
+    if (peak_kv_out) *peak_kv_out = peak;
+    return PS_OK;
+}
+
+ps_status ps_chunk_next(const int32_t* remaining, int32_t n, int32_t budget, int32_t used, int32_t dynamic, int32_t* chunk_out) {
+    ps::clear_error();
+    if (n < 0 || (n > 0 && (!remaining || !chunk_out))) return fail(PS_ERR_INVALID, "ps_chunk_next: n = %d with a null pointer", n);
+    if (budget < 1 || used < 0) return fail(PS_ERR_INVALID, "ps_chunk_next: budget %d, used %d", budget, used);
+    for (int32_t i = 0; i < n; ++i)
+        if (remaining[i] < 1) return fail(PS_ERR_INVALID, "ps_chunk_next: remaining[%d] = %d", i, remaining[i]);
+    int64_t left = (int64_t)budget - used;
+    int32_t i = 0;
+    for (; i < n && left > 0; ++i) {
+        if (dynamic && remaining[i] < 2 * (int64_t)budget) {
+            chunk_out[i] = remaining[i];  // finished at once; the iteration is closed behind it
+            ++i;
+            break;
+        }
+        chunk_out[i] = (int32_t)std::min<int64_t>(remaining[i], left);
+        left -= chunk_out[i];
+    }
+    for (; i < n; ++i) chunk_out[i] = 0;
+    return PS_OK;
+}
+
+ps_status ps_chunk_schedule(int32_t prompt_len, int32_t budget, int32_t first_free, int32_t dynamic, int32_t* chunks_out,
+                            int32_t capacity, int32_t* n_chunks_out) {
+    ps::clear_error();
+    if (!n_chunks_out || (capacity > 0 && !chunks_out) || capacity < 0) return fail(PS_ERR_INVALID, "ps_chunk_schedule: null pointer");
+    if (prompt_len < 1 || budget < 1 || first_free < 0 || first_free > budget)
+        return fail(PS_ERR_INVALID, "ps_chunk_schedule: prompt_len %d, budget %d, first_free %d", prompt_len, budget, first_free);
+    int32_t n = 0, rem = prompt_len, used = budget - first_free;
+    while (rem > 0) {
+        int32_t c = 0;
+        ps_status st = ps_chunk_next(&rem, 1, budget, used, dynamic, &c);
+        if (st) return st;
+        if (c > 0) {
+            if (n < capacity) chunks_out[n] = c;
+            ++n;
+            rem -= c;
+        }
+        used = 0;
+    }
+    *n_chunks_out = n;
+    if (n > capacity) return fail(PS_ERR_INVALID, "ps_chunk_schedule: %d chunks do not fit a capacity of %d", n, capacity);
+    return PS_OK;
+}
+
+ps_status ps_chunk_predict(const ps_table* table, const int32_t* kv_len, const int32_t* remaining, int32_t n_running,
+                           int32_t prompt_len, int32_t max_chunk, double tpot_us, int32_t* chunk_out, int32_t* n_iters_out,
+                           double* completion_us_out, int32_t* maintained_out) {
+    ps::clear_error();
+    if (!table || !chunk_out || !n_iters_out || !completion_us_out || !maintained_out) return fail(PS_ERR_INVALID, "ps_chunk_predict: null pointer");
+    if (prompt_len < 1 || max_chunk < 1) return fail(PS_ERR_INVALID, "ps_chunk_predict: prompt_len %d, max_chunk %d", prompt_len, max_chunk);
+    if (ps_status st = ps::check_requests(kv_len, remaining, n_running)) return st;
+    const ps::Future fut(kv_len, remaining, n_running);
+    const int64_t kv0 = fut.kv(0, 0);
+    int32_t chunk = 0;
+    for (int32_t c = std::min(prompt_len, max_chunk); c >= 1; --c)
+        if (ps::predict(*table, n_running + c, kv0 + c) <= tpot_us) {
+            chunk = c;
+            break;
+        }
+    *chunk_out = chunk;
+    *n_iters_out = 0;
+    *completion_us_out = 0.0;
+    *maintained_out = 0;
+    if (chunk == 0) return PS_OK;
+    const int32_t iters = (int32_t)(((int64_t)prompt_len + chunk - 1) / chunk);
+    double total = 0.0;
+    bool kept = true;
+    size_t pos = 0;
+    for (int32_t k = 0; k < iters; ++k) {
+        pos = fut.first_alive(k, pos);
+        const int64_t alive = (int64_t)n_running - (int64_t)pos;
+        const int64_t done = std::min<int64_t>((int64_t)(k + 1) * chunk, prompt_len);
+        const int64_t c_k = std::min<int64_t>(chunk, (int64_t)prompt_len - (int64_t)k * chunk);
+        const double pred = ps::predict(*table, (int32_t)(alive + c_k), fut.kv(pos, k) + done);
+        total += pred;
+        kept = kept && pred <= tpot_us;
+    }
+    *n_iters_out = iters;
+    *completion_us_out = total;
+    *maintained_out = kept ? 1 : 0;
+    return PS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,170 @@
+"""Scheduler-side entry points (include/polyserve_sched.h) through the C ABI against oracle/sched_oracle.py.
+
+Host code on both sides, so these run without a GPU.  Integers must agree exactly; predicted times to 1e-12
+relative (both sides work in fp64 on the same formula; only the summation order of the fit may differ)."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2507_17769_b200 as ps
+from paper_2507_17769_b200 import binding as B
+from paper_2507_17769_b200 import sched_binding as S
+from oracle import sched_oracle as so
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+REL = 1e-12
+
+
+def test_library_exports_every_symbol_of_the_sched_header():
+    header = open(os.path.join(ROOT, "include", "polyserve_sched.h")).read()
+    declared = set(re.findall(r"\b(ps_[a-z_]+)\s*\(", header)) - {"ps_profile_grid"}  # named in prose only
+    assert declared == set(S.EXPORTS)
+    lib = B.load()
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def grid_rows(rng, batches, per_line=27):
+    rows, plain = [], []
+    for b in batches:
+        a, s = float(rng.uniform(10, 400)), float(rng.uniform(5e-5, 5e-4))
+        for _ in range(per_line):
+            kv = int(rng.integers(1000, 3_000_000))
+            lat = np.float32((a + s * kv) * (1.0 + 0.03 * rng.standard_normal()))
+            r = ps.ps_grid_row()
+            r.token_batch, r.kv_tokens, r.latency_us = b, kv, float(lat)
+            rows.append(r)
+            plain.append((b, kv, float(lat)))
+    order = rng.permutation(len(rows))  # rows of one line need not be adjacent
+    return [rows[i] for i in order], [plain[i] for i in order]
+
+
+def close(a, b):
+    return abs(a - b) <= REL * max(1.0, abs(a), abs(b))
+
+
+def test_table_build_and_predict_match_the_oracle():
+    rng = np.random.default_rng(21)
+    rows, plain = grid_rows(rng, [72, 96, 192, 320, 1032, 2304])
+    t = S.ps_table_build(rows)
+    try:
+        want = so.table_build(plain)
+        b, a, s = S.ps_table_get_lines(t)
+        assert b.tolist() == [ln[0] for ln in want]
+        for i, ln in enumerate(want):
+            assert abs(a[i] - ln[1]) <= 1e-9 * max(1.0, abs(ln[1])) and abs(s[i] - ln[2]) <= 1e-9 * abs(ln[2])
+        lines = list(zip(b.tolist(), a.tolist(), s.tolist()))  # the lookup is compared on the library's own lines
+        for _ in range(2000):
+            tb, kv = int(rng.integers(1, 4000)), int(rng.integers(0, 5_000_000))
+            assert close(S.ps_table_predict(t, tb, kv), so.table_predict(lines, tb, kv))
+        for tb in (1, 72, 73, 95, 96, 2303, 2304, 2305, 10 ** 6):  # at, next to and beyond the lines
+            assert close(S.ps_table_predict(t, tb, 12345), so.table_predict(lines, tb, 12345))
+    finally:
+        S.ps_table_free(t)
+
+
+def test_table_rejects_bad_input():
+    with pytest.raises(ps.PsError):
+        S.ps_table_from_lines([10, 10], [1.0, 2.0], [0.1, 0.1])  # duplicate batch size
+    with pytest.raises(ps.PsError):
+        S.ps_table_from_lines([0], [1.0], [0.1])
+    with pytest.raises(ps.PsError):
+        S.ps_table_from_lines([5], [float("nan")], [0.1])
+    r = ps.ps_grid_row()
+    r.token_batch, r.kv_tokens, r.latency_us = 8, -1, 1.0
+    with pytest.raises(ps.PsError):
+        S.ps_table_build([r])
+    t = S.ps_table_from_lines([5], [1.0], [0.1])
+    with pytest.raises(ps.PsError):
+        S.ps_table_predict(t, 0, 10)
+    with pytest.raises(ps.PsError):
+        S.ps_table_predict(t, 1, -10)
+    S.ps_table_free(t)
+
+
+def random_requests(rng, n, max_len=40000, max_rem=2000):
+    return rng.integers(1, max_len, n).astype(np.int32), rng.integers(1, max_rem, n).astype(np.int32)
+
+
+def test_peak_kv_matches_the_simulation():
+    rng = np.random.default_rng(22)
+    for n in [1, 2, 3, 7, 64, 256]:
+        for _ in range(20):
+            kv, rem = random_requests(rng, n, max_rem=400)
+            assert S.ps_peak_kv(kv, rem) == so.peak_kv(kv.tolist(), rem.tolist())
+    # ties and equal remaining lengths
+    assert S.ps_peak_kv([10, 3], [4, 1]) == (13, 0)
+    assert S.ps_peak_kv([5, 5, 5], [9, 9, 9]) == so.peak_kv([5, 5, 5], [9, 9, 9])
+    assert S.ps_peak_kv([], []) == (0, 0)
+    with pytest.raises(ps.PsError):
+        S.ps_peak_kv([5, 0], [3, 3])
+    with pytest.raises(ps.PsError):
+        S.ps_peak_kv([5, 5], [3, 0])
+
+
+def test_admission_matches_the_oracle():
+    rng = np.random.default_rng(23)
+    lines = [(8, 14.0, 2.2e-4), (64, 16.0, 2.4e-4), (256, 30.0, 2.5e-4), (512, 55.0, 2.6e-4)]
+    t = S.ps_table_from_lines(*zip(*lines))
+    try:
+        flips = 0
+        for _ in range(300):
+            n = int(rng.integers(0, 300))
+            kv, rem = random_requests(rng, n, max_len=9000, max_rem=600)
+            new_kv, new_rem, extra = int(rng.integers(1, 9000)), int(rng.integers(1, 600)), int(rng.integers(0, 3) * 512)
+            tpot = float(rng.uniform(20.0, 500.0))
+            got = S.ps_admit(t, kv, rem, new_kv, new_rem, extra, tpot)
+            want = so.admit(lines, kv.tolist(), rem.tolist(), new_kv, new_rem, extra, tpot)
+            assert got[0] == want[0] and close(got[1], want[1]) and got[2] == want[2]
+            flips += got[0]
+        assert 20 < flips < 280  # both answers occur
+    finally:
+        S.ps_table_free(t)
+
+
+def test_chunk_next_and_schedule_match_the_oracle_and_the_papers_example():
+    assert S.ps_chunk_schedule(2050, 1024, 1024, False).tolist() == [1024, 1024, 2]
+    assert S.ps_chunk_schedule(2050, 1024, 1, False).tolist() == [1, 1024, 1024, 1]
+    assert S.ps_chunk_schedule(2050, 1024, 1024, True).tolist() == [1024, 1026]
+    rng = np.random.default_rng(24)
+    for _ in range(500):
+        budget = int(rng.integers(1, 3000))
+        n = int(rng.integers(0, 12))
+        rem = rng.integers(1, 5 * budget + 2, n).astype(np.int32)
+        used = int(rng.integers(0, budget + 3))
+        for dyn in (False, True):
+            assert S.ps_chunk_next(rem, budget, used, dyn).tolist() == so.chunk_next(rem.tolist(), budget, used, dyn)
+        prompt, free = int(rng.integers(1, 9 * budget + 2)), int(rng.integers(0, budget + 1))
+        for dyn in (False, True):
+            assert S.ps_chunk_schedule(prompt, budget, free, dyn).tolist() == so.chunk_schedule(prompt, budget, free, dyn)
+    with pytest.raises(ps.PsError):
+        S.ps_chunk_next([5], 0, 0, True)
+    with pytest.raises(ps.PsError):
+        S.ps_chunk_next([0], 8, 0, True)
+    with pytest.raises(ps.PsError):
+        S.ps_chunk_schedule(100, 8, 9, False)
+    with pytest.raises(ps.PsError):
+        S.ps_chunk_schedule(100, 8, 8, False, capacity=3)  # 13 chunks do not fit
+
+
+def test_chunk_prediction_matches_the_oracle():
+    rng = np.random.default_rng(25)
+    lines = [(8, 14.0, 2.2e-4), (64, 16.0, 2.4e-4), (256, 30.0, 2.5e-4), (512, 55.0, 2.6e-4), (1024, 100.0, 2.6e-4),
+             (2304, 260.0, 2.7e-4)]
+    t = S.ps_table_from_lines(*zip(*lines))
+    try:
+        seen = set()
+        for _ in range(300):
+            n = int(rng.integers(0, 200))
+            kv, rem = random_requests(rng, n, max_len=6000, max_rem=40)
+            prompt, cap = int(rng.integers(1, 20000)), int(rng.choice([64, 512, 2048, 100000]))
+            tpot = float(rng.uniform(15.0, 900.0))
+            got = S.ps_chunk_predict(t, kv, rem, prompt, cap, tpot)
+            want = so.chunk_predict(lines, kv.tolist(), rem.tolist(), prompt, cap, tpot)
+            assert got[0] == want[0] and got[1] == want[1] and close(got[2], want[2]) and got[3] == want[3]
+            seen.add((got[0] > 0, got[3]))
+        assert seen == {(False, False), (True, False), (True, True)}
+    finally:
+        S.ps_table_free(t)
