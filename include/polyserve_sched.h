@@ -10,9 +10,15 @@
  *     chosen now be kept until the prompt is done?  (section 4.7, "dynamic
  *     chunking" and "continuous chunked prefill prediction")
  * These entry points answer them from a table built out of the rows that
- * ps_profile_grid emits.  They are plain host code: no device is touched, no
- * stream is taken, and they may be called from any thread (a table is
- * immutable once built).  They live in the same shared library as the
+ * ps_profile_grid emits.  The table follows the paper's model of an iteration
+ * (section 3.4): a term that depends on the token batch size, decode attention
+ * as a function of the KV-cache size, and prefill attention as a function of
+ * the prefill work; section 4.5 drops the third term for prompts below 10 K
+ * tokens, here it is kept as an optional coefficient because the profiled
+ * step is attention alone, where a large chunk is not negligible.
+ *
+ * All of this is plain host code: no device is touched, no stream is taken,
+ * and the calls may come from any thread (a table is immutable once built).  They live in the same shared library as the
  * attention entry points and report errors the same way (ps_status,
  * ps_last_error).
  *
@@ -33,7 +39,12 @@
 extern "C" {
 #endif
 
-typedef struct ps_table ps_table; /* (token batch, KV tokens) -> microseconds */
+typedef struct ps_table ps_table; /* (token batch, KV tokens, prefill work) -> microseconds */
+
+/* Prefill-attention work of one chunk of c tokens on `prior` earlier tokens, in
+ * the unit of ps_grid_row.prefill_flops: 4 d Hq (c prior + c (c + 1) / 2). */
+#define PS_PREFILL_FLOPS(head_dim, n_q_heads, c, prior) \
+    (4.0 * (double)(head_dim) * (double)(n_q_heads) * ((double)(c) * (double)(prior) + 0.5 * (double)(c) * ((double)(c) + 1.0)))
 
 /* ------------------------------------------------------------------------ */
 /* Latency table (section 4.5).                                               */
@@ -42,12 +53,16 @@ typedef struct ps_table ps_table; /* (token batch, KV tokens) -> microseconds */
 /*
  * Build a table from n_rows sweep rows (host array, e.g. the output of
  * ps_profile_grid).  Rows with the same token_batch form one line of the
- * table; a line's latency as a function of kv_tokens is the ordinary
- * least-squares straight line through its rows' (kv_tokens, latency_us)
- * points -- iteration time is modelled as affine in the KV-cache size at a
- * fixed batch size (section 3.4: decode attention time is a function of the
- * total number of KV tokens).  A line whose rows all have the same kv_tokens
- * gets slope 0 and their mean latency.  Lines are kept sorted by token_batch.
+ * table: the ordinary least-squares fit
+ *     latency_us = intercept + slope_kv * kv_tokens + slope_pf * prefill_flops
+ * over the line's rows (section 3.4: decode attention time is a function of
+ * the total number of KV tokens, prefill attention of the prefill work; the
+ * intercept carries whatever depends on the batch size alone).  With
+ * centred sums Sxx, Spp, Sxp of the two regressors: if Spp = 0 (no chunk, or
+ * the same work in every row) the line is fitted on kv_tokens alone with
+ * slope_pf = 0; if Sxx = 0 on prefill_flops alone; if both vanish the line is
+ * the mean latency; if the two are collinear (Sxx Spp - Sxp^2 <= 1e-9 Sxx
+ * Spp) on kv_tokens alone.  Lines are kept sorted by token_batch.
  * Errors: PS_ERR_INVALID (null pointers, n_rows < 1, a row with
  * token_batch < 1, kv_tokens < 0 or a latency that is not finite),
  * PS_ERR_OOM.
@@ -56,11 +71,13 @@ ps_status ps_table_build(const ps_grid_row *rows, int64_t n_rows, ps_table **out
 
 /*
  * Build a table from explicit lines: line i predicts intercept_us[i] +
- * slope_us_per_token[i] * kv_tokens at batch size token_batch[i].  The lines
+ * slope_us_per_token[i] * kv_tokens + slope_us_per_flop[i] * prefill_flops at
+ * batch size token_batch[i] (slope_us_per_flop == NULL: all zero).  The lines
  * may come in any order; two lines with the same token_batch are an error.
  */
 ps_status ps_table_from_lines(const int32_t *token_batch, const double *intercept_us,
-                              const double *slope_us_per_token, int32_t n_lines, ps_table **out);
+                              const double *slope_us_per_token, const double *slope_us_per_flop, int32_t n_lines,
+                              ps_table **out);
 
 ps_status ps_table_free(ps_table *table);
 
@@ -68,18 +85,21 @@ ps_status ps_table_free(ps_table *table);
  * be NULL; capacity in lines). */
 ps_status ps_table_size(const ps_table *table, int32_t *n_lines_out);
 ps_status ps_table_get_lines(const ps_table *table, int32_t *token_batch_out, double *intercept_us_out,
-                             double *slope_us_per_token_out, int32_t capacity);
+                             double *slope_us_per_token_out, double *slope_us_per_flop_out, int32_t capacity);
 
 /*
  * Predicted iteration time in microseconds for a batch of token_batch tokens
  * (decode rows count one token each, a prefill chunk its length) whose rows
- * hold kv_tokens tokens of K/V in total.  Between two lines the two lines'
- * values at kv_tokens are interpolated linearly in token_batch; below the
- * first line and above the last one the nearest line is used as it is (no
+ * hold kv_tokens tokens of K/V in total (the chunk's row included) and whose
+ * chunks amount to prefill_flops of attention work (PS_PREFILL_FLOPS summed
+ * over the chunks; 0 for a decode-only batch).  Between two lines the two
+ * lines' values are interpolated linearly in token_batch; below the first
+ * line and above the last one the nearest line is used as it is (no
  * extrapolation in the batch size).  Errors: PS_ERR_INVALID (null pointers,
- * token_batch < 1, kv_tokens < 0).
+ * token_batch < 1, kv_tokens < 0, prefill_flops < 0 or not finite).
  */
-ps_status ps_table_predict(const ps_table *table, int32_t token_batch, int64_t kv_tokens, double *latency_us_out);
+ps_status ps_table_predict(const ps_table *table, int32_t token_batch, int64_t kv_tokens, double prefill_flops,
+                           double *latency_us_out);
 
 /* ------------------------------------------------------------------------ */
 /* Decode admission (section 4.5).                                            */
@@ -101,13 +121,16 @@ ps_status ps_peak_kv(const int32_t *kv_len, const int32_t *remaining, int32_t n,
  * instance running n_running requests: the peak KV-cache size of the running
  * set plus the new request is looked up in the table at the current token
  * batch size (n_running + 1 + extra_tokens; extra_tokens >= 0 counts prefill
- * tokens batched alongside), and the request is admitted when the predicted
- * iteration time is below tpot_us.  Outputs (each may be NULL): *admit_out 1
- * or 0, the predicted time, and the peak KV size used.
+ * tokens batched alongside, extra_kv_tokens >= 0 the K/V their rows hold and
+ * extra_prefill_flops >= 0 their attention work), and the request is admitted
+ * when the predicted iteration time is below tpot_us.  Outputs (each may be
+ * NULL): *admit_out 1 or 0, the predicted time, and the decode requests' peak
+ * KV size (extra_kv_tokens not included).
  */
 ps_status ps_admit(const ps_table *table, const int32_t *kv_len, const int32_t *remaining, int32_t n_running,
-                   int32_t new_kv_len, int32_t new_remaining, int32_t extra_tokens, double tpot_us,
-                   int32_t *admit_out, double *predicted_us_out, int64_t *peak_kv_out);
+                   int32_t new_kv_len, int32_t new_remaining, int32_t extra_tokens, int64_t extra_kv_tokens,
+                   double extra_prefill_flops, double tpot_us, int32_t *admit_out, double *predicted_us_out,
+                   int64_t *peak_kv_out);
 
 /* ------------------------------------------------------------------------ */
 /* Prefill chunking (section 4.7).                                            */
@@ -151,19 +174,24 @@ ps_status ps_chunk_schedule(int32_t prompt_len, int32_t budget, int32_t first_fr
  * tpot_us.  The chunk size predicted at scheduling time is the largest c in
  * [1, min(prompt_len, max_chunk)] for which the table predicts at most tpot_us
  * for iteration 0 (token batch = decode requests alive + c, KV tokens = their
- * KV + c); 0 if there is none.  The prefill then takes ceil(prompt_len / c)
- * iterations; in iteration k the decode requests still alive have grown by k
- * tokens each and the prompt's row holds min((k + 1) c, prompt_len) tokens.
+ * KV + c, prefill work = flops_per_pair c (c + 1) / 2 with flops_per_pair =
+ * 4 head_dim n_q_heads); 0 if there is none.  The prefill
+ * then takes ceil(prompt_len / c) iterations; in iteration k the decode
+ * requests still alive have grown by k tokens each, the prompt's row holds
+ * min((k + 1) c, prompt_len) tokens and its chunk of c_k tokens works on k c
+ * prior tokens.
  * *maintained_out is 1 when every one of those iterations is still predicted
  * at or below tpot_us with that same chunk size (the paper admits the request
  * only then), *completion_us_out the sum of the predicted iteration times (the
  * completion-time estimate to compare with the TTFT), *n_iters_out the number
  * of iterations.  With *chunk_out == 0 the other outputs are 0.
- * Errors: PS_ERR_INVALID (prompt_len < 1, max_chunk < 1, bad request arrays).
+ * Errors: PS_ERR_INVALID (prompt_len < 1, max_chunk < 1, flops_per_pair < 0,
+ * bad request arrays).
  */
 ps_status ps_chunk_predict(const ps_table *table, const int32_t *kv_len, const int32_t *remaining, int32_t n_running,
-                           int32_t prompt_len, int32_t max_chunk, double tpot_us, int32_t *chunk_out,
-                           int32_t *n_iters_out, double *completion_us_out, int32_t *maintained_out);
+                           int32_t prompt_len, int32_t max_chunk, double flops_per_pair, double tpot_us,
+                           int32_t *chunk_out, int32_t *n_iters_out, double *completion_us_out,
+                           int32_t *maintained_out);
 
 #ifdef __cplusplus
 }

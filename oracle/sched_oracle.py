@@ -22,31 +22,46 @@ from __future__ import annotations
 # latency table (section 4.5: a profiled map of (batch size, KV cache size) to execution time)
 # ---------------------------------------------------------------------------
 def table_build(rows):
-    """rows: iterable of (token_batch, kv_tokens, latency_us).  Returns the table as a list of lines
-    (token_batch, intercept_us, slope_us_per_token) sorted by token_batch: per batch size the ordinary
-    least-squares straight line of latency over KV tokens (iteration time is affine in the KV-cache
-    size at a fixed batch size, section 3.4)."""
+    """rows: iterable of (token_batch, kv_tokens, prefill_flops, latency_us).  Returns the table as a list of
+    lines (token_batch, intercept_us, slope_us_per_token, slope_us_per_flop) sorted by token_batch: per batch
+    size the ordinary least-squares fit latency = intercept + slope_kv kv_tokens + slope_pf prefill_flops
+    (section 3.4: an iteration is a batch-size term plus decode attention, a function of the KV-cache size, plus
+    prefill attention, a function of the prefill work).  Normal equations on centred sums; a regressor that does
+    not vary within the line, or the second of two collinear ones, is left out (slope 0)."""
     groups = {}
-    for b, kv, lat in rows:
-        groups.setdefault(int(b), []).append((float(kv), float(lat)))
+    for b, kv, pf, lat in rows:
+        groups.setdefault(int(b), []).append((float(kv), float(pf), float(lat)))
     lines = []
     for b in sorted(groups):
         pts = groups[b]
         n = len(pts)
-        mean_x = sum(x for x, _ in pts) / n
-        mean_y = sum(y for _, y in pts) / n
-        sxx = sum((x - mean_x) * (x - mean_x) for x, _ in pts)
-        sxy = sum((x - mean_x) * (y - mean_y) for x, y in pts)
-        slope = sxy / sxx if sxx > 0.0 else 0.0
-        lines.append((b, mean_y - slope * mean_x, slope))
+        mx = sum(x for x, _, _ in pts) / n
+        mp = sum(q for _, q, _ in pts) / n
+        my = sum(y for _, _, y in pts) / n
+        sxx = sum((x - mx) * (x - mx) for x, _, _ in pts)
+        spp = sum((q - mp) * (q - mp) for _, q, _ in pts)
+        sxp = sum((x - mx) * (q - mp) for x, q, _ in pts)
+        sxy = sum((x - mx) * (y - my) for x, _, y in pts)
+        spy = sum((q - mp) * (y - my) for _, q, y in pts)
+        det = sxx * spp - sxp * sxp
+        if sxx > 0.0 and spp > 0.0 and det > 1e-9 * sxx * spp:
+            s_kv = (sxy * spp - spy * sxp) / det
+            s_pf = (spy * sxx - sxy * sxp) / det
+        elif sxx > 0.0:
+            s_kv, s_pf = sxy / sxx, 0.0
+        elif spp > 0.0:
+            s_kv, s_pf = 0.0, spy / spp
+        else:
+            s_kv, s_pf = 0.0, 0.0
+        lines.append((b, my - s_kv * mx - s_pf * mp, s_kv, s_pf))
     return lines
 
 
-def table_predict(lines, token_batch, kv_tokens):
-    """Predicted iteration time: the line of that batch size evaluated at kv_tokens; between two lines their
-    two values interpolated linearly in the batch size; outside the lines the nearest line as it is."""
+def table_predict(lines, token_batch, kv_tokens, prefill_flops=0.0):
+    """Predicted iteration time: the line of that batch size evaluated at (kv_tokens, prefill_flops); between two
+    lines their two values interpolated linearly in the batch size; outside the lines the nearest line as it is."""
     lines = sorted(lines)
-    at = lambda ln: ln[1] + ln[2] * float(kv_tokens)
+    at = lambda ln: ln[1] + ln[2] * float(kv_tokens) + ln[3] * float(prefill_flops)
     if token_batch <= lines[0][0]:
         return at(lines[0])
     if token_batch >= lines[-1][0]:
@@ -78,12 +93,13 @@ def peak_kv(kv_len, remaining):
     return peak, when
 
 
-def admit(lines, kv_len, remaining, new_kv_len, new_remaining, extra_tokens, tpot_us):
-    """(admitted?, predicted iteration time, peak KV) for one new decode request: the table at the current
-    token batch size and the largest future KV-cache size must stay below the TPOT."""
+def admit(lines, kv_len, remaining, new_kv_len, new_remaining, extra_tokens, extra_kv_tokens, extra_prefill_flops, tpot_us):
+    """(admitted?, predicted iteration time, peak KV of the decode requests) for one new decode request: the table
+    at the current token batch size and the largest future KV-cache size must stay below the TPOT.  Prefill
+    tokens batched alongside add their tokens, the K/V of their rows and their attention work to the lookup."""
     peak, _ = peak_kv(list(kv_len) + [new_kv_len], list(remaining) + [new_remaining])
     batch = len(kv_len) + 1 + extra_tokens
-    pred = table_predict(lines, batch, peak)
+    pred = table_predict(lines, batch, peak + extra_kv_tokens, extra_prefill_flops)
     return pred < tpot_us, pred, peak
 
 
@@ -118,12 +134,17 @@ def chunk_schedule(prompt_len, budget, first_free, dynamic):
     return chunks
 
 
-def chunk_predict(lines, kv_len, remaining, prompt_len, max_chunk, tpot_us):
+def prefill_work(flops_per_pair, c, prior):
+    """Attention work of a chunk of c tokens on `prior` earlier ones: token i sees prior + i + 1 keys."""
+    return flops_per_pair * (float(c) * float(prior) + 0.5 * float(c) * (float(c) + 1.0))
+
+
+def chunk_predict(lines, kv_len, remaining, prompt_len, max_chunk, flops_per_pair, tpot_us):
     """Continuous chunked-prefill prediction.  Returns (chunk, iterations, completion_us, maintained)."""
     kv0, n0 = kv_at(kv_len, remaining, 0)
     chunk = 0
     for c in range(min(prompt_len, max_chunk), 0, -1):
-        if table_predict(lines, n0 + c, kv0 + c) <= tpot_us:
+        if table_predict(lines, n0 + c, kv0 + c, prefill_work(flops_per_pair, c, 0)) <= tpot_us:
             chunk = c
             break
     if chunk == 0:
@@ -133,7 +154,7 @@ def chunk_predict(lines, kv_len, remaining, prompt_len, max_chunk, tpot_us):
     for k in range(iters):
         kv, n = kv_at(kv_len, remaining, k)
         c_k = min(chunk, prompt_len - k * chunk)
-        pred = table_predict(lines, n + c_k, kv + min((k + 1) * chunk, prompt_len))
+        pred = table_predict(lines, n + c_k, kv + min((k + 1) * chunk, prompt_len), prefill_work(flops_per_pair, c_k, k * chunk))
         completion += pred
         maintained = maintained and pred <= tpot_us
     return chunk, iters, completion, maintained

@@ -13,23 +13,26 @@
 struct ps_table {
     std::vector<int32_t> batch;   // sorted, distinct
     std::vector<double> intercept;
-    std::vector<double> slope;
+    std::vector<double> slope;     // microseconds per KV token
+    std::vector<double> slope_pf;  // microseconds per flop of prefill attention
 };
 
 namespace ps {
 namespace {
 
-double line_at(const ps_table& t, size_t i, int64_t kv) { return t.intercept[i] + t.slope[i] * (double)kv; }
+double line_at(const ps_table& t, size_t i, int64_t kv, double pf) {
+    return t.intercept[i] + t.slope[i] * (double)kv + t.slope_pf[i] * pf;
+}
 
-double predict(const ps_table& t, int32_t token_batch, int64_t kv) {
+double predict(const ps_table& t, int32_t token_batch, int64_t kv, double pf) {
     const size_t n = t.batch.size();
-    if (token_batch <= t.batch.front()) return line_at(t, 0, kv);
-    if (token_batch >= t.batch.back()) return line_at(t, n - 1, kv);
+    if (token_batch <= t.batch.front()) return line_at(t, 0, kv, pf);
+    if (token_batch >= t.batch.back()) return line_at(t, n - 1, kv, pf);
     // lines lo, hi with batch[lo] <= token_batch < batch[hi]
     const size_t hi = (size_t)(std::upper_bound(t.batch.begin(), t.batch.end(), token_batch) - t.batch.begin());
     const size_t lo = hi - 1;
     const double w = (double)(token_batch - t.batch[lo]) / (double)(t.batch[hi] - t.batch[lo]);
-    const double a = line_at(t, lo, kv), b = line_at(t, hi, kv);
+    const double a = line_at(t, lo, kv, pf), b = line_at(t, hi, kv, pf);
     return a + (b - a) * w;
 }
 
@@ -75,6 +78,11 @@ struct Future {
     }
 };
 
+// attention work of a chunk of c tokens on `prior` earlier ones
+double prefill_work(double flops_per_pair, int64_t c, int64_t prior) {
+    return flops_per_pair * ((double)c * (double)prior + 0.5 * (double)c * ((double)c + 1.0));
+}
+
 }  // namespace
 }  // namespace ps
 
@@ -83,7 +91,7 @@ using ps::fail;
 extern "C" {
 
 ps_status ps_table_from_lines(const int32_t* token_batch, const double* intercept_us, const double* slope_us_per_token,
-                              int32_t n_lines, ps_table** out) {
+                              const double* slope_us_per_flop, int32_t n_lines, ps_table** out) {
     ps::clear_error();
     if (!token_batch || !intercept_us || !slope_us_per_token || !out || n_lines < 1)
         return fail(PS_ERR_INVALID, "ps_table_from_lines: null pointer or n_lines < 1");
@@ -94,7 +102,8 @@ ps_status ps_table_from_lines(const int32_t* token_batch, const double* intercep
     if (!t) return fail(PS_ERR_OOM, "ps_table_from_lines: out of host memory");
     for (int32_t k = 0; k < n_lines; ++k) {
         const int32_t i = order[k];
-        if (token_batch[i] < 1 || !std::isfinite(intercept_us[i]) || !std::isfinite(slope_us_per_token[i]) ||
+        const double pf_slope = slope_us_per_flop ? slope_us_per_flop[i] : 0.0;
+        if (token_batch[i] < 1 || !std::isfinite(intercept_us[i]) || !std::isfinite(slope_us_per_token[i]) || !std::isfinite(pf_slope) ||
             (k > 0 && token_batch[i] == token_batch[order[k - 1]])) {
             delete t;
             return fail(PS_ERR_INVALID, "ps_table_from_lines: line %d (token_batch %d) is not usable or is a duplicate", i, token_batch[i]);
@@ -102,6 +111,7 @@ ps_status ps_table_from_lines(const int32_t* token_batch, const double* intercep
         t->batch.push_back(token_batch[i]);
         t->intercept.push_back(intercept_us[i]);
         t->slope.push_back(slope_us_per_token[i]);
+        t->slope_pf.push_back(pf_slope);
     }
     *out = t;
     return PS_OK;
@@ -111,7 +121,8 @@ ps_status ps_table_build(const ps_grid_row* rows, int64_t n_rows, ps_table** out
     ps::clear_error();
     if (!rows || !out || n_rows < 1) return fail(PS_ERR_INVALID, "ps_table_build: null pointer or n_rows < 1");
     for (int64_t i = 0; i < n_rows; ++i)
-        if (rows[i].token_batch < 1 || rows[i].kv_tokens < 0 || !std::isfinite(rows[i].latency_us))
+        if (rows[i].token_batch < 1 || rows[i].kv_tokens < 0 || !std::isfinite(rows[i].latency_us) || !std::isfinite(rows[i].prefill_flops) ||
+            rows[i].prefill_flops < 0.0)
             return fail(PS_ERR_INVALID, "ps_table_build: row %lld has token_batch %d, kv_tokens %lld, latency %g", (long long)i,
                         rows[i].token_batch, (long long)rows[i].kv_tokens, (double)rows[i].latency_us);
     // rows of one batch size together, in their input order
@@ -119,27 +130,42 @@ ps_status ps_table_build(const ps_grid_row* rows, int64_t n_rows, ps_table** out
     std::iota(order.begin(), order.end(), (int64_t)0);
     std::stable_sort(order.begin(), order.end(), [&](int64_t a, int64_t b) { return rows[a].token_batch < rows[b].token_batch; });
     std::vector<int32_t> batch;
-    std::vector<double> icpt, slope;
+    std::vector<double> icpt, slope, slope_pf;
     for (int64_t g0 = 0; g0 < n_rows;) {
         int64_t g1 = g0;
         while (g1 < n_rows && rows[order[g1]].token_batch == rows[order[g0]].token_batch) ++g1;
         const double n = (double)(g1 - g0);
-        double sum_x = 0.0, sum_y = 0.0;
-        for (int64_t k = g0; k < g1; ++k) sum_x += (double)rows[order[k]].kv_tokens, sum_y += (double)rows[order[k]].latency_us;
-        const double mean_x = sum_x / n, mean_y = sum_y / n;
-        double sxx = 0.0, sxy = 0.0;
+        double sum_x = 0.0, sum_p = 0.0, sum_y = 0.0;
         for (int64_t k = g0; k < g1; ++k) {
-            const double dx = (double)rows[order[k]].kv_tokens - mean_x;
-            sxx += dx * dx;
-            sxy += dx * ((double)rows[order[k]].latency_us - mean_y);
+            const ps_grid_row& r = rows[order[k]];
+            sum_x += (double)r.kv_tokens, sum_p += r.prefill_flops, sum_y += (double)r.latency_us;
         }
-        const double s = sxx > 0.0 ? sxy / sxx : 0.0;
+        const double mx = sum_x / n, mp = sum_p / n, my = sum_y / n;
+        double sxx = 0.0, spp = 0.0, sxp = 0.0, sxy = 0.0, spy = 0.0;
+        for (int64_t k = g0; k < g1; ++k) {
+            const ps_grid_row& r = rows[order[k]];
+            const double dx = (double)r.kv_tokens - mx, dp = r.prefill_flops - mp, dy = (double)r.latency_us - my;
+            sxx += dx * dx, spp += dp * dp, sxp += dx * dp, sxy += dx * dy, spy += dp * dy;
+        }
+        // normal equations of latency = a + s kv + q pf on centred sums; a regressor that does not vary within the
+        // line, or the second of two collinear ones, is left out
+        const double det = sxx * spp - sxp * sxp;
+        double s_kv = 0.0, s_pf = 0.0;
+        if (sxx > 0.0 && spp > 0.0 && det > 1e-9 * sxx * spp) {
+            s_kv = (sxy * spp - spy * sxp) / det;
+            s_pf = (spy * sxx - sxy * sxp) / det;
+        } else if (sxx > 0.0) {
+            s_kv = sxy / sxx;
+        } else if (spp > 0.0) {
+            s_pf = spy / spp;
+        }
         batch.push_back(rows[order[g0]].token_batch);
-        slope.push_back(s);
-        icpt.push_back(mean_y - s * mean_x);
+        slope.push_back(s_kv);
+        slope_pf.push_back(s_pf);
+        icpt.push_back(my - s_kv * mx - s_pf * mp);
         g0 = g1;
     }
-    return ps_table_from_lines(batch.data(), icpt.data(), slope.data(), (int32_t)batch.size(), out);
+    return ps_table_from_lines(batch.data(), icpt.data(), slope.data(), slope_pf.data(), (int32_t)batch.size(), out);
 }
 
 ps_status ps_table_free(ps_table* table) {
@@ -155,7 +181,7 @@ ps_status ps_table_size(const ps_table* table, int32_t* n_lines_out) {
 }
 
 ps_status ps_table_get_lines(const ps_table* table, int32_t* token_batch_out, double* intercept_us_out,
-                             double* slope_us_per_token_out, int32_t capacity) {
+                             double* slope_us_per_token_out, double* slope_us_per_flop_out, int32_t capacity) {
     ps::clear_error();
     if (!table) return fail(PS_ERR_INVALID, "ps_table_get_lines: null table");
     if (capacity < (int32_t)table->batch.size()) return fail(PS_ERR_INVALID, "ps_table_get_lines: capacity %d < %zu lines", capacity, table->batch.size());
@@ -163,15 +189,17 @@ ps_status ps_table_get_lines(const ps_table* table, int32_t* token_batch_out, do
         if (token_batch_out) token_batch_out[i] = table->batch[i];
         if (intercept_us_out) intercept_us_out[i] = table->intercept[i];
         if (slope_us_per_token_out) slope_us_per_token_out[i] = table->slope[i];
+        if (slope_us_per_flop_out) slope_us_per_flop_out[i] = table->slope_pf[i];
     }
     return PS_OK;
 }
 
-ps_status ps_table_predict(const ps_table* table, int32_t token_batch, int64_t kv_tokens, double* latency_us_out) {
+ps_status ps_table_predict(const ps_table* table, int32_t token_batch, int64_t kv_tokens, double prefill_flops, double* latency_us_out) {
     ps::clear_error();
     if (!table || !latency_us_out) return fail(PS_ERR_INVALID, "ps_table_predict: null pointer");
-    if (token_batch < 1 || kv_tokens < 0) return fail(PS_ERR_INVALID, "ps_table_predict: token_batch %d, kv_tokens %lld", token_batch, (long long)kv_tokens);
-    *latency_us_out = ps::predict(*table, token_batch, kv_tokens);
+    if (token_batch < 1 || kv_tokens < 0 || !(prefill_flops >= 0.0) || !std::isfinite(prefill_flops))
+        return fail(PS_ERR_INVALID, "ps_table_predict: token_batch %d, kv_tokens %lld, prefill_flops %g", token_batch, (long long)kv_tokens, prefill_flops);
+    *latency_us_out = ps::predict(*table, token_batch, kv_tokens, prefill_flops);
     return PS_OK;
 }
 
@@ -184,11 +212,13 @@ ps_status ps_peak_kv(const int32_t* kv_len, const int32_t* remaining, int32_t n,
 }
 
 ps_status ps_admit(const ps_table* table, const int32_t* kv_len, const int32_t* remaining, int32_t n_running, int32_t new_kv_len,
-                   int32_t new_remaining, int32_t extra_tokens, double tpot_us, int32_t* admit_out, double* predicted_us_out,
-                   int64_t* peak_kv_out) {
+                   int32_t new_remaining, int32_t extra_tokens, int64_t extra_kv_tokens, double extra_prefill_flops, double tpot_us,
+                   int32_t* admit_out, double* predicted_us_out, int64_t* peak_kv_out) {
     ps::clear_error();
     if (!table) return fail(PS_ERR_INVALID, "ps_admit: null table");
-    if (extra_tokens < 0) return fail(PS_ERR_INVALID, "ps_admit: extra_tokens %d < 0", extra_tokens);
+    if (extra_tokens < 0 || extra_kv_tokens < 0 || !(extra_prefill_flops >= 0.0) || !std::isfinite(extra_prefill_flops))
+        return fail(PS_ERR_INVALID, "ps_admit: extra_tokens %d, extra_kv_tokens %lld, extra_prefill_flops %g", extra_tokens,
+                    (long long)extra_kv_tokens, extra_prefill_flops);
     if (ps_status st = ps::check_requests(kv_len, remaining, n_running)) return st;
     if (ps_status st = ps::check_requests(&new_kv_len, &new_remaining, 1)) return st;
     std::vector<int32_t> len(kv_len, kv_len + n_running), rem(remaining, remaining + n_running);
@@ -197,7 +227,7 @@ ps_status ps_admit(const ps_table* table, const int32_t* kv_len, const int32_t* 
     int64_t peak = 0;
     int32_t when = 0;
     ps::Future(len.data(), rem.data(), n_running + 1).peak(&peak, &when);
-    const double pred = ps::predict(*table, n_running + 1 + extra_tokens, peak);
+    const double pred = ps::predict(*table, n_running + 1 + extra_tokens, peak + extra_kv_tokens, extra_prefill_flops);
     if (admit_out) *admit_out = pred < tpot_us ? 1 : 0;
     if (predicted_us_out) *predicted_us_out = pred;
     if (peak_kv_out) *peak_kv_out = peak;
@@ -249,17 +279,18 @@ ps_status ps_chunk_schedule(int32_t prompt_len, int32_t budget, int32_t first_fr
 }
 
 ps_status ps_chunk_predict(const ps_table* table, const int32_t* kv_len, const int32_t* remaining, int32_t n_running,
-                           int32_t prompt_len, int32_t max_chunk, double tpot_us, int32_t* chunk_out, int32_t* n_iters_out,
-                           double* completion_us_out, int32_t* maintained_out) {
+                           int32_t prompt_len, int32_t max_chunk, double flops_per_pair, double tpot_us, int32_t* chunk_out,
+                           int32_t* n_iters_out, double* completion_us_out, int32_t* maintained_out) {
     ps::clear_error();
     if (!table || !chunk_out || !n_iters_out || !completion_us_out || !maintained_out) return fail(PS_ERR_INVALID, "ps_chunk_predict: null pointer");
-    if (prompt_len < 1 || max_chunk < 1) return fail(PS_ERR_INVALID, "ps_chunk_predict: prompt_len %d, max_chunk %d", prompt_len, max_chunk);
+    if (prompt_len < 1 || max_chunk < 1 || !(flops_per_pair >= 0.0) || !std::isfinite(flops_per_pair))
+        return fail(PS_ERR_INVALID, "ps_chunk_predict: prompt_len %d, max_chunk %d, flops_per_pair %g", prompt_len, max_chunk, flops_per_pair);
     if (ps_status st = ps::check_requests(kv_len, remaining, n_running)) return st;
     const ps::Future fut(kv_len, remaining, n_running);
     const int64_t kv0 = fut.kv(0, 0);
     int32_t chunk = 0;
     for (int32_t c = std::min(prompt_len, max_chunk); c >= 1; --c)
-        if (ps::predict(*table, n_running + c, kv0 + c) <= tpot_us) {
+        if (ps::predict(*table, n_running + c, kv0 + c, ps::prefill_work(flops_per_pair, c, 0)) <= tpot_us) {
             chunk = c;
             break;
         }
@@ -277,7 +308,7 @@ ps_status ps_chunk_predict(const ps_table* table, const int32_t* kv_len, const i
         const int64_t alive = (int64_t)n_running - (int64_t)pos;
         const int64_t done = std::min<int64_t>((int64_t)(k + 1) * chunk, prompt_len);
         const int64_t c_k = std::min<int64_t>(chunk, (int64_t)prompt_len - (int64_t)k * chunk);
-        const double pred = ps::predict(*table, (int32_t)(alive + c_k), fut.kv(pos, k) + done);
+        const double pred = ps::predict(*table, (int32_t)(alive + c_k), fut.kv(pos, k) + done, ps::prefill_work(flops_per_pair, c_k, (int64_t)k * chunk));
         total += pred;
         kept = kept && pred <= tpot_us;
     }

@@ -24,17 +24,17 @@ def _lib():
     lib = B.load()
     if not _ready:
         lib.ps_table_build.argtypes = [ctypes.POINTER(B.ps_grid_row), _i64, ctypes.POINTER(_vp)]
-        lib.ps_table_from_lines.argtypes = [_i32p, _f64p, _f64p, _i32, ctypes.POINTER(_vp)]
+        lib.ps_table_from_lines.argtypes = [_i32p, _f64p, _f64p, _f64p, _i32, ctypes.POINTER(_vp)]
         lib.ps_table_free.argtypes = [_vp]
         lib.ps_table_size.argtypes = [_vp, ctypes.POINTER(_i32)]
-        lib.ps_table_get_lines.argtypes = [_vp, _i32p, _f64p, _f64p, _i32]
-        lib.ps_table_predict.argtypes = [_vp, _i32, _i64, _f64p]
+        lib.ps_table_get_lines.argtypes = [_vp, _i32p, _f64p, _f64p, _f64p, _i32]
+        lib.ps_table_predict.argtypes = [_vp, _i32, _i64, _f64, _f64p]
         lib.ps_peak_kv.argtypes = [_i32p, _i32p, _i32, ctypes.POINTER(_i64), ctypes.POINTER(_i32)]
-        lib.ps_admit.argtypes = [_vp, _i32p, _i32p, _i32, _i32, _i32, _i32, _f64, ctypes.POINTER(_i32), _f64p,
+        lib.ps_admit.argtypes = [_vp, _i32p, _i32p, _i32, _i32, _i32, _i32, _i64, _f64, _f64, ctypes.POINTER(_i32), _f64p,
                                  ctypes.POINTER(_i64)]
         lib.ps_chunk_next.argtypes = [_i32p, _i32, _i32, _i32, _i32, _i32p]
         lib.ps_chunk_schedule.argtypes = [_i32, _i32, _i32, _i32, _i32p, _i32, ctypes.POINTER(_i32)]
-        lib.ps_chunk_predict.argtypes = [_vp, _i32p, _i32p, _i32, _i32, _i32, _f64, ctypes.POINTER(_i32),
+        lib.ps_chunk_predict.argtypes = [_vp, _i32p, _i32p, _i32, _i32, _i32, _f64, _f64, ctypes.POINTER(_i32),
                                          ctypes.POINTER(_i32), _f64p, ctypes.POINTER(_i32)]
         for name in EXPORTS:
             getattr(lib, name).restype = ctypes.c_int
@@ -55,12 +55,13 @@ def ps_table_build(rows):
     return out.value
 
 
-def ps_table_from_lines(token_batch, intercept_us, slope_us_per_token):
+def ps_table_from_lines(token_batch, intercept_us, slope_us_per_token, slope_us_per_flop=None):
     b, bp = B._host_i32(token_batch)
     a, ap = _host_f64(intercept_us)
     s, sp = _host_f64(slope_us_per_token)
+    q, qp = _host_f64(slope_us_per_flop) if slope_us_per_flop is not None else (None, None)
     out = _vp(0)
-    B._check(_lib().ps_table_from_lines(bp, ap, sp, b.shape[0], ctypes.byref(out)))
+    B._check(_lib().ps_table_from_lines(bp, ap, sp, qp, b.shape[0], ctypes.byref(out)))
     return out.value
 
 
@@ -75,16 +76,17 @@ def ps_table_size(table) -> int:
 
 
 def ps_table_get_lines(table):
-    """Returns (token_batch int32[n], intercept_us float64[n], slope_us_per_token float64[n]), sorted by batch size."""
+    """Returns (token_batch int32[n], intercept_us, slope_us_per_token, slope_us_per_flop: float64[n]), sorted by batch size."""
     n = ps_table_size(table)
-    b, a, s = np.zeros(n, np.int32), np.zeros(n, np.float64), np.zeros(n, np.float64)
-    B._check(_lib().ps_table_get_lines(table, b.ctypes.data_as(_i32p), a.ctypes.data_as(_f64p), s.ctypes.data_as(_f64p), n))
-    return b, a, s
+    b, a, s, q = np.zeros(n, np.int32), np.zeros(n, np.float64), np.zeros(n, np.float64), np.zeros(n, np.float64)
+    B._check(_lib().ps_table_get_lines(table, b.ctypes.data_as(_i32p), a.ctypes.data_as(_f64p), s.ctypes.data_as(_f64p),
+                                       q.ctypes.data_as(_f64p), n))
+    return b, a, s, q
 
 
-def ps_table_predict(table, token_batch: int, kv_tokens: int) -> float:
+def ps_table_predict(table, token_batch: int, kv_tokens: int, prefill_flops: float = 0.0) -> float:
     out = _f64(0.0)
-    B._check(_lib().ps_table_predict(table, token_batch, kv_tokens, ctypes.byref(out)))
+    B._check(_lib().ps_table_predict(table, token_batch, kv_tokens, prefill_flops, ctypes.byref(out)))
     return out.value
 
 
@@ -97,12 +99,13 @@ def ps_peak_kv(kv_len, remaining):
     return peak.value, when.value
 
 
-def ps_admit(table, kv_len, remaining, new_kv_len, new_remaining, extra_tokens, tpot_us):
-    """Returns (admitted: bool, predicted_us, peak_kv)."""
+def ps_admit(table, kv_len, remaining, new_kv_len, new_remaining, extra_tokens, extra_kv_tokens, extra_prefill_flops, tpot_us):
+    """Returns (admitted: bool, predicted_us, peak_kv of the decode requests)."""
     kv, kvp = B._host_i32(kv_len)
     rm, rmp = B._host_i32(remaining)
     ok, pred, peak = _i32(0), _f64(0.0), _i64(0)
-    B._check(_lib().ps_admit(table, kvp, rmp, kv.shape[0], new_kv_len, new_remaining, extra_tokens, tpot_us,
+    B._check(_lib().ps_admit(table, kvp, rmp, kv.shape[0], new_kv_len, new_remaining, extra_tokens, extra_kv_tokens,
+                             extra_prefill_flops, tpot_us,
                              ctypes.byref(ok), ctypes.byref(pred), ctypes.byref(peak)))
     return bool(ok.value), pred.value, peak.value
 
@@ -122,11 +125,11 @@ def ps_chunk_schedule(prompt_len, budget, first_free, dynamic, capacity=None):
     return out[: n.value]
 
 
-def ps_chunk_predict(table, kv_len, remaining, prompt_len, max_chunk, tpot_us):
+def ps_chunk_predict(table, kv_len, remaining, prompt_len, max_chunk, flops_per_pair, tpot_us):
     """Returns (chunk, iterations, completion_us, maintained: bool)."""
     kv, kvp = B._host_i32(kv_len)
     rm, rmp = B._host_i32(remaining)
     c, it, tot, kept = _i32(0), _i32(0), _f64(0.0), _i32(0)
-    B._check(_lib().ps_chunk_predict(table, kvp, rmp, kv.shape[0], prompt_len, max_chunk, tpot_us, ctypes.byref(c),
+    B._check(_lib().ps_chunk_predict(table, kvp, rmp, kv.shape[0], prompt_len, max_chunk, flops_per_pair, tpot_us, ctypes.byref(c),
                                      ctypes.byref(it), ctypes.byref(tot), ctypes.byref(kept)))
     return c.value, it.value, tot.value, bool(kept.value)

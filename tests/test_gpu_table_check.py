@@ -15,15 +15,15 @@ def test_table_from_a_sweep_predicts_held_out_decode_heavy_batches():
     rows = ps.ps_profile_grid(shape, (64, 256), (32, 128), (1024, 4096), 3, 2, 5, 3000)
     table = S.ps_table_build(rows)
     try:
-        b, icpt, slope = S.ps_table_get_lines(table)
+        b, icpt, slope, slope_pf = S.ps_table_get_lines(table)
         assert b.tolist() == [96, 192, 288, 384] and (slope > 0).all()   # more KV tokens cost more time
         held = ps.ps_profile_grid(shape, (128,), (64,), (2048,), 3, 2, 5, 9000)
         err = rel_errors(table, held)
         assert np.median(np.abs(err)) < 0.5
         # admission flips from yes to no as the TPOT tightens around the predicted time
         kv, rem = np.full(63, 2048, np.int32), np.full(63, 100, np.int32)
-        ok, pred, peak = S.ps_admit(table, kv, rem, 2048, 100, 0, 1e9)
+        ok, pred, peak = S.ps_admit(table, kv, rem, 2048, 100, 0, 0, 0.0, 1e9)
         assert ok and peak == 64 * (2048 + 99)
-        assert not S.ps_admit(table, kv, rem, 2048, 100, 0, pred * 0.99)[0]
+        assert not S.ps_admit(table, kv, rem, 2048, 100, 0, 0, 0.0, pred * 0.99)[0]
     finally:
         S.ps_table_free(table)

@@ -112,28 +112,58 @@ def test_peak_kv_monotone_in_the_request_set():
 def test_table_fit_recovers_exact_lines_and_matches_numpy():
     rng = np.random.default_rng(3)
     rows = []
-    truth = {72: (15.0, 2.5e-4), 320: (40.0, 3.0e-4), 2304: (310.0, 1.0e-4)}
-    for b, (a, s) in truth.items():
+    truth = {72: (15.0, 2.5e-4, 0.0), 320: (40.0, 3.0e-4, 0.0), 2304: (310.0, 1.0e-4, 0.0)}
+    for b, (a, s, _) in truth.items():
         for kv in rng.integers(1000, 2_000_000, 27):
-            rows.append((b, int(kv), a + s * float(kv)))
+            rows.append((b, int(kv), 0.0, a + s * float(kv)))   # no chunk: the prefill regressor does not vary
     lines = so.table_build(rows)
     assert [ln[0] for ln in lines] == sorted(truth)
-    for b, a, s in lines:
-        assert abs(a - truth[b][0]) < 1e-6 and abs(s - truth[b][1]) < 1e-12
+    for b, a, s, q in lines:
+        assert abs(a - truth[b][0]) < 1e-6 and abs(s - truth[b][1]) < 1e-12 and q == 0.0
     # noisy data: the same coefficients as numpy's least squares
-    noisy = [(b, kv, lat * (1.0 + 0.05 * rng.standard_normal())) for b, kv, lat in rows]
-    for b, a, s in so.table_build(noisy):
-        x = np.array([kv for bb, kv, _ in noisy if bb == b], dtype=np.float64)
-        y = np.array([lat for bb, _, lat in noisy if bb == b], dtype=np.float64)
+    noisy = [(b, kv, pf, lat * (1.0 + 0.05 * rng.standard_normal())) for b, kv, pf, lat in rows]
+    for b, a, s, q in so.table_build(noisy):
+        x = np.array([kv for bb, kv, _, _ in noisy if bb == b], dtype=np.float64)
+        y = np.array([lat for bb, _, _, lat in noisy if bb == b], dtype=np.float64)
         coef, *_ = np.linalg.lstsq(np.stack([np.ones_like(x), x], axis=1), y, rcond=None)
         assert abs(a - coef[0]) < 1e-6 * max(1.0, abs(coef[0])) and abs(s - coef[1]) < 1e-9 * abs(coef[1])
     # a line whose rows share one KV size: slope 0 and their mean
-    flat = so.table_build([(8, 500, 10.0), (8, 500, 14.0)])
-    assert flat == [(8, 12.0, 0.0)]
+    flat = so.table_build([(8, 500, 0.0, 10.0), (8, 500, 0.0, 14.0)])
+    assert flat == [(8, 12.0, 0.0, 0.0)]
+
+
+def test_table_fit_with_the_prefill_term():
+    rng = np.random.default_rng(4)
+    # exact planes are recovered
+    rows, truth = [], {1032: (42.0, 6.0e-4, 1.1e-9), 2056: (60.0, 6.5e-4, 0.9e-9)}
+    for b, (a, s, q) in truth.items():
+        for _ in range(27):
+            kv, pf = int(rng.integers(10_000, 300_000)), float(rng.uniform(1e9, 4e11))
+            rows.append((b, kv, pf, a + s * kv + q * pf))
+    for b, a, s, q in so.table_build(rows):
+        assert abs(a - truth[b][0]) < 1e-6 and abs(s - truth[b][1]) < 1e-12 and abs(q - truth[b][2]) < 1e-18
+    # noisy: numpy's least squares on [1, kv, pf] (columns scaled for its conditioning), and residual orthogonal to the regressors
+    noisy = [(b, kv, pf, lat * (1.0 + 0.05 * rng.standard_normal())) for b, kv, pf, lat in rows]
+    for b, a, s, q in so.table_build(noisy):
+        x = np.array([kv for bb, kv, _, _ in noisy if bb == b], dtype=np.float64)
+        w = np.array([pf for bb, _, pf, _ in noisy if bb == b], dtype=np.float64)
+        y = np.array([lat for bb, _, _, lat in noisy if bb == b], dtype=np.float64)
+        coef, *_ = np.linalg.lstsq(np.stack([np.ones_like(x), x / 1e5, w / 1e11], axis=1), y, rcond=None)
+        assert abs(a - coef[0]) < 1e-6 * max(1.0, abs(coef[0]))
+        assert abs(s - coef[1] / 1e5) < 1e-8 * abs(coef[1] / 1e5) and abs(q - coef[2] / 1e11) < 1e-8 * abs(coef[2] / 1e11)
+        res = y - (a + s * x + q * w)
+        assert abs(res.sum()) < 1e-6 * np.abs(y).sum() and abs((res * (x - x.mean())).sum()) < 1e-6 * np.abs(y * x).sum()
+        assert abs((res * (w - w.mean())).sum()) < 1e-6 * np.abs(y * w).sum()
+    # collinear regressors: the prefill term is left out, the KV line is fitted alone
+    col = so.table_build([(520, kv, 3.0e5 * kv, 20.0 + 7e-4 * kv) for kv in (1000, 2000, 5000, 9000)])
+    assert col[0][3] == 0.0 and abs(col[0][2] - 7e-4) < 1e-12 and abs(col[0][1] - 20.0) < 1e-9
+    # only the prefill work varies
+    pf_only = so.table_build([(520, 4000, pf, 30.0 + 1e-9 * pf) for pf in (1e9, 5e9, 2e10)])
+    assert pf_only[0][2] == 0.0 and abs(pf_only[0][3] - 1e-9) < 1e-18 and abs(pf_only[0][1] - 30.0) < 1e-9
 
 
 def test_table_lookup_interpolates_in_batch_and_clamps():
-    lines = [(100, 10.0, 1e-3), (300, 50.0, 2e-3)]
+    lines = [(100, 10.0, 1e-3, 0.0), (300, 50.0, 2e-3, 1e-9)]
     assert so.table_predict(lines, 100, 1000) == pytest.approx(11.0)
     assert so.table_predict(lines, 300, 1000) == pytest.approx(52.0)
     assert so.table_predict(lines, 200, 1000) == pytest.approx(0.5 * (11.0 + 52.0))   # midpoint
@@ -141,43 +171,59 @@ def test_table_lookup_interpolates_in_batch_and_clamps():
     assert so.table_predict(lines, 5, 1000) == pytest.approx(11.0)                   # below: first line
     assert so.table_predict(lines, 9000, 1000) == pytest.approx(52.0)                # above: last line
     assert so.table_predict(list(reversed(lines)), 200, 1000) == pytest.approx(31.5)  # order of the lines is free
+    # the prefill work enters through each line's own coefficient
+    assert so.table_predict(lines, 300, 1000, 4e9) == pytest.approx(56.0)
+    assert so.table_predict(lines, 100, 1000, 4e9) == pytest.approx(11.0)
+    assert so.table_predict(lines, 200, 1000, 4e9) == pytest.approx(0.5 * (11.0 + 56.0))
 
 
 def test_admission_uses_the_peak_and_the_current_batch_size():
     # table(b, kv) = 2 b + 0.01 kv
-    lines = [(1, 2.0, 0.01), (1001, 2002.0, 0.01)]
+    lines = [(1, 2.0, 0.01, 1e-9), (1001, 2002.0, 0.01, 1e-9)]
     kv, rem = [100, 200], [10, 3]
     # with the newcomer (50 tokens, 5 to go): t0 = 350, t1 = 353, t2 = 356, t3 = 103+53 = 156, t4 = 158 -> peak 356
-    ok, pred, peak = so.admit(lines, kv, rem, 50, 5, 0, 10.0)
+    ok, pred, peak = so.admit(lines, kv, rem, 50, 5, 0, 0, 0.0, 10.0)
     assert peak == 356 and pred == pytest.approx(2 * 3 + 3.56) and ok
-    assert not so.admit(lines, kv, rem, 50, 5, 0, 9.56)[0]          # strictly below the TPOT is required
-    assert so.admit(lines, kv, rem, 50, 5, 0, 9.5601)[0]
-    # prefill tokens batched alongside count in the batch size only
-    ok, pred, peak = so.admit(lines, kv, rem, 50, 5, 100, 1e9)
+    assert not so.admit(lines, kv, rem, 50, 5, 0, 0, 0.0, 9.56)[0]          # strictly below the TPOT is required
+    assert so.admit(lines, kv, rem, 50, 5, 0, 0, 0.0, 9.5601)[0]
+    # prefill tokens batched alongside: their tokens, the K/V of their rows and their attention work join the lookup
+    ok, pred, peak = so.admit(lines, kv, rem, 50, 5, 100, 0, 0.0, 1e9)
     assert peak == 356 and pred == pytest.approx(2 * 103 + 3.56)
+    ok, pred, peak = so.admit(lines, kv, rem, 50, 5, 100, 1100, 3e9, 1e9)
+    assert peak == 356 and pred == pytest.approx(2 * 103 + 0.01 * (356 + 1100) + 3.0)
 
 
 def test_chunk_prediction_closed_form():
     # table(b, kv) = alpha b + beta kv, no decode requests: chunk c costs (alpha + beta) c in iteration 0
     alpha, beta = 0.1, 0.002
-    lines = [(1, alpha, beta), (100001, alpha * 100001, beta)]
+    lines = [(1, alpha, beta, 0.0), (100001, alpha * 100001, beta, 0.0)]
     tpot = 50.0
-    c, iters, total, kept = so.chunk_predict(lines, [], [], 3000, 2048, tpot)
+    c, iters, total, kept = so.chunk_predict(lines, [], [], 3000, 2048, 16384.0, tpot)
     assert c == int(tpot / (alpha + beta))                       # 490
     assert iters == -(-3000 // c)
     # iteration k costs alpha c_k + beta min((k + 1) c, P); it grows with k, so the chunk size is not kept
     want = sum(alpha * min(c, 3000 - k * c) + beta * min((k + 1) * c, 3000) for k in range(iters))
     assert total == pytest.approx(want) and not kept
     # with beta = 0 the cost does not grow: the chunk is kept
-    lines0 = [(1, alpha, 0.0), (100001, alpha * 100001, 0.0)]
-    c, iters, total, kept = so.chunk_predict(lines0, [], [], 3000, 2048, tpot)
+    lines0 = [(1, alpha, 0.0, 0.0), (100001, alpha * 100001, 0.0, 0.0)]
+    c, iters, total, kept = so.chunk_predict(lines0, [], [], 3000, 2048, 16384.0, tpot)
     assert c == 500 and iters == 6 and kept and total == pytest.approx(alpha * 3000)
     # decode requests take their share: alpha (n + c) + beta (KV + c) <= tpot
     kv, rem = [1000] * 20, [1000] * 20
-    c, *_ = so.chunk_predict(lines, kv, rem, 3000, 2048, tpot)
+    c, *_ = so.chunk_predict(lines, kv, rem, 3000, 2048, 16384.0, tpot)
     assert c == int((tpot - alpha * 20 - beta * 20000) / (alpha + beta) + 1e-9)
     # no chunk fits
-    assert so.chunk_predict(lines, [10 ** 6], [5], 100, 2048, tpot) == (0, 0, 0.0, False)
+    assert so.chunk_predict(lines, [10 ** 6], [5], 100, 2048, 16384.0, tpot) == (0, 0, 0.0, False)
     # the cap and the prompt length bound the chunk
-    assert so.chunk_predict(lines0, [], [], 3000, 128, tpot)[0] == 128
-    assert so.chunk_predict(lines0, [], [], 77, 2048, tpot)[:2] == (77, 1)
+    assert so.chunk_predict(lines0, [], [], 3000, 128, 16384.0, tpot)[0] == 128
+    assert so.chunk_predict(lines0, [], [], 77, 2048, 16384.0, tpot)[:2] == (77, 1)
+    # a table with a prefill term only: iteration 0 costs g phi c (c + 1) / 2, so c is the root of a quadratic;
+    # later chunks work on k c prior tokens and cost more, so the size is not kept past the first
+    g, phi = 1e-9, 16384.0
+    lines_pf = [(1, 0.0, 0.0, g), (100001, 0.0, 0.0, g)]
+    c, iters, total, kept = so.chunk_predict(lines_pf, [], [], 5000, 4096, phi, tpot)
+    root = int((-1.0 + (1.0 + 8.0 * tpot / (g * phi)) ** 0.5) / 2.0)
+    assert c == root and iters == -(-5000 // c) and not kept
+    want = sum(g * phi * (min(c, 5000 - k * c) * k * c + 0.5 * min(c, 5000 - k * c) * (min(c, 5000 - k * c) + 1)) for k in range(iters))
+    assert total == pytest.approx(want)
+    assert so.prefill_work(4.0 * 128 * 32, 1536, 3885) == 4 * 128 * 32 * (1536 * 3885 + 1536 * 1537 // 2)

@@ -29,14 +29,16 @@ def test_library_exports_every_symbol_of_the_sched_header():
 def grid_rows(rng, batches, per_line=27):
     rows, plain = [], []
     for b in batches:
-        a, s = float(rng.uniform(10, 400)), float(rng.uniform(5e-5, 5e-4))
+        a, s, q = float(rng.uniform(10, 400)), float(rng.uniform(5e-5, 5e-4)), float(rng.uniform(5e-10, 2e-9))
+        with_chunk = b != batches[0]  # the first line is decode-only: its prefill work is 0 in every row
         for _ in range(per_line):
             kv = int(rng.integers(1000, 3_000_000))
-            lat = np.float32((a + s * kv) * (1.0 + 0.03 * rng.standard_normal()))
+            pf = float(rng.uniform(1e9, 5e11)) if with_chunk else 0.0
+            lat = np.float32((a + s * kv + q * pf) * (1.0 + 0.03 * rng.standard_normal()))
             r = ps.ps_grid_row()
-            r.token_batch, r.kv_tokens, r.latency_us = b, kv, float(lat)
+            r.token_batch, r.kv_tokens, r.prefill_flops, r.latency_us = b, kv, pf, float(lat)
             rows.append(r)
-            plain.append((b, kv, float(lat)))
+            plain.append((b, kv, pf, float(lat)))
     order = rng.permutation(len(rows))  # rows of one line need not be adjacent
     return [rows[i] for i in order], [plain[i] for i in order]
 
@@ -51,18 +53,37 @@ def test_table_build_and_predict_match_the_oracle():
     t = S.ps_table_build(rows)
     try:
         want = so.table_build(plain)
-        b, a, s = S.ps_table_get_lines(t)
+        b, a, s, q = S.ps_table_get_lines(t)
         assert b.tolist() == [ln[0] for ln in want]
         for i, ln in enumerate(want):
             assert abs(a[i] - ln[1]) <= 1e-9 * max(1.0, abs(ln[1])) and abs(s[i] - ln[2]) <= 1e-9 * abs(ln[2])
-        lines = list(zip(b.tolist(), a.tolist(), s.tolist()))  # the lookup is compared on the library's own lines
+            assert abs(q[i] - ln[3]) <= 1e-9 * abs(ln[3]) and (q[i] != 0.0) == (i > 0)
+        lines = list(zip(b.tolist(), a.tolist(), s.tolist(), q.tolist()))  # the lookup is compared on the library's own lines
         for _ in range(2000):
-            tb, kv = int(rng.integers(1, 4000)), int(rng.integers(0, 5_000_000))
-            assert close(S.ps_table_predict(t, tb, kv), so.table_predict(lines, tb, kv))
+            tb, kv, pf = int(rng.integers(1, 4000)), int(rng.integers(0, 5_000_000)), float(rng.uniform(0, 6e11))
+            assert close(S.ps_table_predict(t, tb, kv, pf), so.table_predict(lines, tb, kv, pf))
         for tb in (1, 72, 73, 95, 96, 2303, 2304, 2305, 10 ** 6):  # at, next to and beyond the lines
-            assert close(S.ps_table_predict(t, tb, 12345), so.table_predict(lines, tb, 12345))
+            assert close(S.ps_table_predict(t, tb, 12345, 1e10), so.table_predict(lines, tb, 12345, 1e10))
     finally:
         S.ps_table_free(t)
+    # degenerate lines: collinear regressors, only the prefill work varying, nothing varying
+    cases = [[(520, kv, 3.0e5 * kv, 20.0 + 7e-4 * kv) for kv in (1000, 2000, 5000, 9000)],
+             [(520, 4000, pf, 30.0 + 1e-9 * pf) for pf in (1e9, 5e9, 2e10)],
+             [(8, 500, 0.0, 10.0), (8, 500, 0.0, 14.0)]]
+    for plain in cases:
+        rows = []
+        for b, kv, pf, lat in plain:
+            r = ps.ps_grid_row()
+            r.token_batch, r.kv_tokens, r.prefill_flops, r.latency_us = b, kv, pf, lat
+            rows.append(r)
+        t = S.ps_table_build(rows)
+        try:
+            got = [x.tolist()[0] for x in S.ps_table_get_lines(t)]
+            want = so.table_build([(b, kv, pf, float(np.float32(lat))) for b, kv, pf, lat in plain])[0]
+            assert got[0] == want[0] and all(abs(g - w) <= 1e-9 * max(1e-12, abs(w)) for g, w in zip(got[1:], want[1:]))
+            assert [g == 0.0 for g in got[2:]] == [w == 0.0 for w in want[2:]]
+        finally:
+            S.ps_table_free(t)
 
 
 def test_table_rejects_bad_input():
@@ -81,6 +102,8 @@ def test_table_rejects_bad_input():
         S.ps_table_predict(t, 0, 10)
     with pytest.raises(ps.PsError):
         S.ps_table_predict(t, 1, -10)
+    with pytest.raises(ps.PsError):
+        S.ps_table_predict(t, 1, 10, -1.0)
     S.ps_table_free(t)
 
 
@@ -106,7 +129,8 @@ def test_peak_kv_matches_the_simulation():
 
 def test_admission_matches_the_oracle():
     rng = np.random.default_rng(23)
-    lines = [(8, 14.0, 2.2e-4), (64, 16.0, 2.4e-4), (256, 30.0, 2.5e-4), (512, 55.0, 2.6e-4)]
+    lines = [(8, 14.0, 2.2e-4, 0.0), (64, 16.0, 2.4e-4, 0.0), (256, 30.0, 2.5e-4, 1.0e-9), (512, 55.0, 2.6e-4, 1.2e-9),
+             (2304, 80.0, 2.6e-4, 1.1e-9)]
     t = S.ps_table_from_lines(*zip(*lines))
     try:
         flips = 0
@@ -114,9 +138,11 @@ def test_admission_matches_the_oracle():
             n = int(rng.integers(0, 300))
             kv, rem = random_requests(rng, n, max_len=9000, max_rem=600)
             new_kv, new_rem, extra = int(rng.integers(1, 9000)), int(rng.integers(1, 600)), int(rng.integers(0, 3) * 512)
+            extra_kv = extra + int(rng.integers(0, 8192)) if extra else 0
+            extra_pf = 4.0 * 128 * 32 * (extra * (extra_kv - extra) + extra * (extra + 1) / 2)
             tpot = float(rng.uniform(20.0, 500.0))
-            got = S.ps_admit(t, kv, rem, new_kv, new_rem, extra, tpot)
-            want = so.admit(lines, kv.tolist(), rem.tolist(), new_kv, new_rem, extra, tpot)
+            got = S.ps_admit(t, kv, rem, new_kv, new_rem, extra, extra_kv, extra_pf, tpot)
+            want = so.admit(lines, kv.tolist(), rem.tolist(), new_kv, new_rem, extra, extra_kv, extra_pf, tpot)
             assert got[0] == want[0] and close(got[1], want[1]) and got[2] == want[2]
             flips += got[0]
         assert 20 < flips < 280  # both answers occur
@@ -151,8 +177,8 @@ def test_chunk_next_and_schedule_match_the_oracle_and_the_papers_example():
 
 def test_chunk_prediction_matches_the_oracle():
     rng = np.random.default_rng(25)
-    lines = [(8, 14.0, 2.2e-4), (64, 16.0, 2.4e-4), (256, 30.0, 2.5e-4), (512, 55.0, 2.6e-4), (1024, 100.0, 2.6e-4),
-             (2304, 260.0, 2.7e-4)]
+    lines = [(8, 14.0, 2.2e-4, 0.0), (64, 16.0, 2.4e-4, 6e-10), (256, 30.0, 2.5e-4, 1.0e-9), (512, 35.0, 2.6e-4, 1.2e-9),
+             (1024, 40.0, 2.6e-4, 1.1e-9), (2304, 60.0, 2.7e-4, 1.0e-9)]
     t = S.ps_table_from_lines(*zip(*lines))
     try:
         seen = set()
@@ -161,8 +187,8 @@ def test_chunk_prediction_matches_the_oracle():
             kv, rem = random_requests(rng, n, max_len=6000, max_rem=40)
             prompt, cap = int(rng.integers(1, 20000)), int(rng.choice([64, 512, 2048, 100000]))
             tpot = float(rng.uniform(15.0, 900.0))
-            got = S.ps_chunk_predict(t, kv, rem, prompt, cap, tpot)
-            want = so.chunk_predict(lines, kv.tolist(), rem.tolist(), prompt, cap, tpot)
+            got = S.ps_chunk_predict(t, kv, rem, prompt, cap, 4.0 * 128 * 32, tpot)
+            want = so.chunk_predict(lines, kv.tolist(), rem.tolist(), prompt, cap, 4.0 * 128 * 32, tpot)
             assert got[0] == want[0] and got[1] == want[1] and close(got[2], want[2]) and got[3] == want[3]
             seen.add((got[0] > 0, got[3]))
         assert seen == {(False, False), (True, False), (True, True)}
