@@ -270,6 +270,8 @@ typedef struct {
     int32_t warmup;               /* untimed runs per draw (>= 1) */
     int32_t iters;                /* timed runs per draw (>= 1) */
     uint64_t seed_base;           /* draw s of cell c uses seed seed_base + seeds_per_cell * c + s */
+    int32_t include_kv_write;     /* != 0: each timed run first appends the batch's new tokens with ps_kv_write
+                                     (section 2.1: the pass that computes attention also populates the cache) */
 } ps_grid_spec;
 
 typedef struct {
@@ -299,7 +301,8 @@ typedef struct {
  * rows (host, capacity max_rows) receives one row per draw in sweep order
  * (chunk-major, then decode count, then mean context, then seed);
  * *n_rows_out is the count written.  If csv_path is not NULL the rows are also
- * written there as CSV with a header line.
+ * written there as CSV with a header line (first column: "attn", or
+ * "attn+kv_write" when the append is inside the timed region).
  * Errors: PS_ERR_INVALID (null/empty spec, max_rows too small),
  * PS_ERR_UNSUPPORTED, PS_ERR_OOM, PS_ERR_CUDA; a device-side error of any run
  * aborts the sweep with that status.

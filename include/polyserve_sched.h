@@ -81,6 +81,21 @@ ps_status ps_table_from_lines(const int32_t *token_batch, const double *intercep
 
 ps_status ps_table_free(ps_table *table);
 
+/*
+ * Add a term that depends on the token batch size alone to every line of the
+ * table -- the GEMM(B) of the paper's iteration model (section 3.4: T_iter =
+ * GEMM(B) + decode attention + prefill attention), measured by the caller for
+ * its model's linear layers.  The term is given at n >= 1 sample batch sizes
+ * (any order, distinct) and interpolated linearly between them; outside the
+ * samples the nearest one is used.  ps_table_scale multiplies every
+ * coefficient by factor > 0 (n identical layers: n times one layer).  Both
+ * change the table in place: call them before sharing it between threads.
+ * Errors: PS_ERR_INVALID (null pointers, n < 1, a batch size < 1 or repeated,
+ * a value that is not finite, factor <= 0).
+ */
+ps_status ps_table_add_batch_term(ps_table *table, const int32_t *token_batch, const double *term_us, int32_t n);
+ps_status ps_table_scale(ps_table *table, double factor);
+
 /* Number of lines; and a copy of them, sorted by token_batch (any output may
  * be NULL; capacity in lines). */
 ps_status ps_table_size(const ps_table *table, int32_t *n_lines_out);

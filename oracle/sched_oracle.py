@@ -73,6 +73,30 @@ def table_predict(lines, token_batch, kv_tokens, prefill_flops=0.0):
     raise AssertionError("unreachable")
 
 
+def table_add_batch_term(lines, samples):
+    """The table with a term that depends on the token batch size alone added to every line (section 3.4: the
+    GEMMs and collectives of an iteration depend on the batch size only).  samples: (token_batch, microseconds)
+    pairs; between two samples the term is interpolated linearly, outside them the nearest sample is used."""
+    samples = sorted(samples)
+
+    def term(b):
+        if b <= samples[0][0]:
+            return samples[0][1]
+        if b >= samples[-1][0]:
+            return samples[-1][1]
+        for lo, hi in zip(samples[:-1], samples[1:]):
+            if lo[0] <= b < hi[0]:
+                return lo[1] + (hi[1] - lo[1]) * ((b - lo[0]) / float(hi[0] - lo[0]))
+        raise AssertionError("unreachable")
+
+    return [(b, a + term(b), s, q) for b, a, s, q in lines]
+
+
+def table_scale(lines, factor):
+    """Every coefficient times factor (a model of n identical layers is n times one layer)."""
+    return [(b, a * factor, s * factor, q * factor) for b, a, s, q in lines]
+
+
 # ---------------------------------------------------------------------------
 # decode admission (section 4.5: simulate future iterations, take the largest KV-cache size)
 # ---------------------------------------------------------------------------

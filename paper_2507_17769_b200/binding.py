@@ -51,7 +51,7 @@ class ps_grid_spec(ctypes.Structure):
                 ("decode_counts", ctypes.POINTER(ctypes.c_int32)), ("n_decode_counts", ctypes.c_int32),
                 ("mean_ctxs", ctypes.POINTER(ctypes.c_int32)), ("n_mean_ctxs", ctypes.c_int32),
                 ("seeds_per_cell", ctypes.c_int32), ("warmup", ctypes.c_int32), ("iters", ctypes.c_int32),
-                ("seed_base", ctypes.c_uint64)]
+                ("seed_base", ctypes.c_uint64), ("include_kv_write", ctypes.c_int32)]
 
 
 class ps_grid_row(ctypes.Structure):
@@ -238,12 +238,13 @@ def ps_plan_get_timing(plan, stream=None):
 
 
 def ps_profile_grid(shape: ps_shape, chunk_sizes, decode_counts, mean_ctxs, seeds_per_cell, warmup, iters, seed_base,
-                    csv_path=None, stream=None):
+                    csv_path=None, stream=None, include_kv_write=False):
     """Returns the list of ps_grid_row in sweep order."""
     ca, cp = _host_i32(chunk_sizes)
     da, dp = _host_i32(decode_counts)
     ma, mp = _host_i32(mean_ctxs)
-    spec = ps_grid_spec(cp, ca.shape[0], dp, da.shape[0], mp, ma.shape[0], seeds_per_cell, warmup, iters, seed_base)
+    spec = ps_grid_spec(cp, ca.shape[0], dp, da.shape[0], mp, ma.shape[0], seeds_per_cell, warmup, iters, seed_base,
+                        int(bool(include_kv_write)))
     n = ca.shape[0] * da.shape[0] * ma.shape[0] * seeds_per_cell
     rows = (ps_grid_row * n)()
     n_out = _i64(0)

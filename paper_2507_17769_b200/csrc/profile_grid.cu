@@ -158,7 +158,7 @@ extern "C" ps_status ps_profile_grid(const ps_shape* shape, const ps_grid_spec* 
                 }
         (void)dr;
     }
-    DevBuf pool_mem, q_mem, out_mem, bt_mem, ws_mem;
+    DevBuf pool_mem, q_mem, out_mem, bt_mem, ws_mem, knew_mem, vnew_mem;
     size_t ws_cap = 0;
     if (pool_mem.alloc((size_t)cap_pages * page_bytes) != cudaSuccess)
         return fail(PS_ERR_OOM, "cannot allocate %zu bytes of KV pool for the sweep", (size_t)cap_pages * page_bytes);
@@ -166,6 +166,13 @@ extern "C" ps_status ps_profile_grid(const ps_shape* shape, const ps_grid_spec* 
     if (q_mem.alloc(q_bytes) != cudaSuccess || out_mem.alloc(q_bytes) != cudaSuccess ||
         bt_mem.alloc((size_t)cap_bt * sizeof(int32_t)) != cudaSuccess)
         return fail(PS_ERR_OOM, "cannot allocate sweep buffers");
+    const size_t new_bytes = (size_t)cap_q * Hkv * d * 2;  // K (or V) of one batch's new tokens
+    if (spec->include_kv_write) {
+        if (knew_mem.alloc(new_bytes) != cudaSuccess || vnew_mem.alloc(new_bytes) != cudaSuccess)
+            return fail(PS_ERR_OOM, "cannot allocate sweep buffers");
+        fill_kernel<<<148, 256, 0, s>>>((uint16_t*)knew_mem.p, (int64_t)(new_bytes / 2), 0x9abc);
+        fill_kernel<<<148, 256, 0, s>>>((uint16_t*)vnew_mem.p, (int64_t)(new_bytes / 2), 0xdef0);
+    }
     fill_kernel<<<148 * 8, 256, 0, s>>>((uint16_t*)pool_mem.p, (int64_t)((size_t)cap_pages * page_bytes / 2), 0x1234);
     fill_kernel<<<148, 256, 0, s>>>((uint16_t*)q_mem.p, (int64_t)(q_bytes / 2), 0x5678);
     PS_CUDA_TRY(cudaGetLastError());
@@ -241,6 +248,10 @@ extern "C" ps_status ps_profile_grid(const ps_shape* shape, const ps_grid_spec* 
                     for (int it = 0; it < n_ev && result == PS_OK; ++it) {
                         const int32_t* bt_k = (const int32_t*)bt_mem.p + (size_t)(it % rot) * dr.block_table.size();
                         cudaEventRecord(ev0[it], s);
+                        if (spec->include_kv_write) {
+                            result = ps_kv_write(kv, knew_mem.p, vnew_mem.p, bt_k, dr.max_pages, dr.prior.data(), dr.q_len.data(), n, s);
+                            if (result != PS_OK) break;
+                        }
                         result = ps_attn_run(plan, kv, q_mem.p, bt_k, out_mem.p, nullptr, ws_mem.p, ws_cap, s);
                         cudaEventRecord(ev1[it], s);
                     }
@@ -272,7 +283,8 @@ extern "C" ps_status ps_profile_grid(const ps_shape* shape, const ps_grid_spec* 
                     r.latency_max_us = times.back();
                     r.plan_us = (float)std::chrono::duration<double, std::micro>(t1 - t0).count();
                     if (csv)
-                        fprintf(csv, "attn,%d,%d,%d,%d,%llu,%d,%d,%lld,%.0f,%.0f,%.3f,%.3f,%.3f,%.3f\n", r.chunk, r.n_decode,
+                        fprintf(csv, "%s,%d,%d,%d,%d,%llu,%d,%d,%lld,%.0f,%.0f,%.3f,%.3f,%.3f,%.3f\n",
+                                spec->include_kv_write ? "attn+kv_write" : "attn", r.chunk, r.n_decode,
                                 r.mean_ctx, r.seed_index, (unsigned long long)r.seed, r.token_batch, r.prefill_prior,
                                 (long long)r.kv_tokens, r.decode_bytes, r.prefill_flops, r.latency_us, r.latency_min_us,
                                 r.latency_max_us, r.plan_us);

@@ -173,6 +173,46 @@ ps_status ps_table_free(ps_table* table) {
     return PS_OK;
 }
 
+ps_status ps_table_add_batch_term(ps_table* table, const int32_t* token_batch, const double* term_us, int32_t n) {
+    ps::clear_error();
+    if (!table || !token_batch || !term_us || n < 1) return fail(PS_ERR_INVALID, "ps_table_add_batch_term: null pointer or n < 1");
+    std::vector<int32_t> order(n);
+    std::iota(order.begin(), order.end(), 0);
+    std::sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return token_batch[a] < token_batch[b]; });
+    for (int32_t k = 0; k < n; ++k) {
+        const int32_t i = order[k];
+        if (token_batch[i] < 1 || !std::isfinite(term_us[i]) || (k > 0 && token_batch[i] == token_batch[order[k - 1]]))
+            return fail(PS_ERR_INVALID, "ps_table_add_batch_term: sample %d (token_batch %d) is not usable or is a duplicate", i, token_batch[i]);
+    }
+    for (size_t l = 0; l < table->batch.size(); ++l) {
+        const int32_t b = table->batch[l];
+        double term;
+        if (b <= token_batch[order.front()]) {
+            term = term_us[order.front()];
+        } else if (b >= token_batch[order.back()]) {
+            term = term_us[order.back()];
+        } else {
+            int32_t k = 0;
+            while (token_batch[order[k + 1]] <= b) ++k;  // samples k, k + 1 with batch[k] <= b < batch[k + 1]
+            const int32_t lo = order[k], hi = order[k + 1];
+            term = term_us[lo] + (term_us[hi] - term_us[lo]) * ((double)(b - token_batch[lo]) / (double)(token_batch[hi] - token_batch[lo]));
+        }
+        table->intercept[l] += term;
+    }
+    return PS_OK;
+}
+
+ps_status ps_table_scale(ps_table* table, double factor) {
+    ps::clear_error();
+    if (!table || !(factor > 0.0) || !std::isfinite(factor)) return fail(PS_ERR_INVALID, "ps_table_scale: null table or factor %g", factor);
+    for (size_t l = 0; l < table->batch.size(); ++l) {
+        table->intercept[l] *= factor;
+        table->slope[l] *= factor;
+        table->slope_pf[l] *= factor;
+    }
+    return PS_OK;
+}
+
 ps_status ps_table_size(const ps_table* table, int32_t* n_lines_out) {
     ps::clear_error();
     if (!table || !n_lines_out) return fail(PS_ERR_INVALID, "ps_table_size: null pointer");

@@ -11,7 +11,8 @@ import numpy as np
 
 from . import binding as B
 
-EXPORTS = ["ps_table_build", "ps_table_from_lines", "ps_table_free", "ps_table_size", "ps_table_get_lines",
+EXPORTS = ["ps_table_build", "ps_table_from_lines", "ps_table_free", "ps_table_add_batch_term", "ps_table_scale", "ps_table_size",
+           "ps_table_get_lines",
            "ps_table_predict", "ps_peak_kv", "ps_admit", "ps_chunk_next", "ps_chunk_schedule", "ps_chunk_predict"]
 
 _vp, _i32, _i64, _f64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_double
@@ -26,6 +27,8 @@ def _lib():
         lib.ps_table_build.argtypes = [ctypes.POINTER(B.ps_grid_row), _i64, ctypes.POINTER(_vp)]
         lib.ps_table_from_lines.argtypes = [_i32p, _f64p, _f64p, _f64p, _i32, ctypes.POINTER(_vp)]
         lib.ps_table_free.argtypes = [_vp]
+        lib.ps_table_add_batch_term.argtypes = [_vp, _i32p, _f64p, _i32]
+        lib.ps_table_scale.argtypes = [_vp, _f64]
         lib.ps_table_size.argtypes = [_vp, ctypes.POINTER(_i32)]
         lib.ps_table_get_lines.argtypes = [_vp, _i32p, _f64p, _f64p, _f64p, _i32]
         lib.ps_table_predict.argtypes = [_vp, _i32, _i64, _f64, _f64p]
@@ -67,6 +70,17 @@ def ps_table_from_lines(token_batch, intercept_us, slope_us_per_token, slope_us_
 
 def ps_table_free(table):
     B._check(_lib().ps_table_free(table))
+
+
+def ps_table_add_batch_term(table, token_batch, term_us):
+    """Adds a batch-size-only term (the model's GEMM time at the sampled batch sizes) to every line, in place."""
+    b, bp = B._host_i32(token_batch)
+    t, tp = _host_f64(term_us)
+    B._check(_lib().ps_table_add_batch_term(table, bp, tp, b.shape[0]))
+
+
+def ps_table_scale(table, factor: float):
+    B._check(_lib().ps_table_scale(table, factor))
 
 
 def ps_table_size(table) -> int:

@@ -9,6 +9,11 @@
    paper's two keys alone (prefill work left out of the fit).  Prints the relative prediction errors.
 3. The host cost of the admission test (ps_admit) and of the chunk prediction (ps_chunk_predict) for an instance
    with 256 running requests, in decisions per second through this binding.
+4. With --iteration: the whole-iteration table of the paper's model T_iter = GEMM(B) + decode attention + prefill
+   attention (section 3.4) for an 8B-class decoder (32 layers, hidden 4096, 32 q / 8 kv heads of 128, FFN 14336): the
+   sweep is repeated with the KV append inside the timed region, the linear layers' time at each of the table's batch
+   sizes is measured with library GEMMs (torch.matmul, bf16; weights of four layers in rotation so that none is found
+   in L2) and added with ps_table_add_batch_term, and everything is scaled to 32 layers with ps_table_scale.
 
 The paper's keys (token batch size, KV-cache size) do not carry the chunk's own prior context, so a table on those
 two alone predicts prefill-heavy batches poorly; the report shows both tables and splits the batches by chunk size.
@@ -68,6 +73,54 @@ def host_rates(table, n_running=256, calls=20000, seed=7):
     return {"n_running": n_running, "admit_per_s": 1.0 / admit_s, "chunk_predict_per_s": 1.0 / chunk_s}
 
 
+LAYERS, HIDDEN, KV_DIM, FFN = 32, 4096, 1024, 14336
+
+
+def layer_gemm_us(batches, reps=20):
+    """Time of one decoder layer's linear layers (QKV, O, gate+up, down) on B tokens, per B, with torch.matmul."""
+    import torch
+
+    dev = torch.device("cuda")
+    shapes = [(HIDDEN, HIDDEN + 2 * KV_DIM), (HIDDEN, HIDDEN), (HIDDEN, 2 * FFN), (FFN, HIDDEN)]
+    weights = [[torch.randn(k, n, device=dev, dtype=torch.bfloat16) * 0.02 for k, n in shapes] for _ in range(4)]
+    out = []
+    for b in batches:
+        xs = [torch.randn(int(b), k, device=dev, dtype=torch.bfloat16) for k, _ in shapes]
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        times = []
+        for it in range(reps + 5):
+            w = weights[it % 4]
+            ev0.record()
+            for x, m in zip(xs, w):
+                torch.matmul(x, m)
+            ev1.record()
+            torch.cuda.synchronize()
+            if it >= 5:
+                times.append(ev0.elapsed_time(ev1) * 1e3)
+        out.append(float(np.median(times)))
+    return out
+
+
+def iteration_table(shape, grid, seeds, warmup, iters):
+    rows = B.ps_profile_grid(shape, *grid, seeds, warmup, iters, 3000, include_kv_write=True)
+    table = S.ps_table_build(rows)
+    b, _, _, _ = S.ps_table_get_lines(table)
+    gemm = layer_gemm_us(b.tolist())
+    S.ps_table_add_batch_term(table, b, gemm)
+    S.ps_table_scale(table, float(LAYERS))
+    print("whole-iteration table (%d layers; per layer: attention with KV append + linear layers):" % LAYERS)
+    for bi, g in zip(b.tolist(), gemm):
+        print("  token_batch %5d: linear layers %8.1f us per layer" % (bi, g))
+    phi = 4.0 * shape.head_dim * shape.n_q_heads
+    for n_dec, ctx, chunk, prior in [(64, 1024, 0, 0), (256, 2048, 0, 0), (256, 8192, 0, 0), (128, 2048, 512, 2048), (256, 2048, 1792, 4096)]:
+        kv = n_dec * ctx + (chunk + prior if chunk else 0)
+        pf = phi * (chunk * prior + 0.5 * chunk * (chunk + 1.0))
+        t = S.ps_table_predict(table, n_dec + chunk, kv, pf)
+        print("  %3d decodes at %5d tokens%s: predicted iteration %.2f ms" %
+              (n_dec, ctx, " + %d-token chunk on %d" % (chunk, prior) if chunk else "", t / 1e3))
+    return table
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--seeds", type=int, default=27)
@@ -76,6 +129,7 @@ def main():
     ap.add_argument("--iters", type=int, default=10)
     ap.add_argument("--quick", action="store_true", help="corner cells of the grid, 3 seeds; two held-out shapes")
     ap.add_argument("--heads", default="32,8,128", help="n_q_heads,n_kv_heads,head_dim")
+    ap.add_argument("--iteration", action="store_true", help="also build the whole-iteration table of an 8B-class model")
     a = ap.parse_args()
     hq, hkv, d = (int(x) for x in a.heads.split(","))
     shape = B.make_shape(hq, hkv, d)
@@ -104,6 +158,8 @@ def main():
         finally:
             S.ps_table_free(blind)
         print(json.dumps(report))
+        if a.iteration:
+            S.ps_table_free(iteration_table(shape, grid, seeds, a.warmup, a.iters))
     finally:
         S.ps_table_free(table)
 

@@ -36,6 +36,18 @@ def test_grid_rows_keys_and_regenerable_lengths(tmp_path):
     assert large > 0.8 * small
 
 
+def test_grid_with_the_kv_append_in_the_timed_region(tmp_path):
+    sh = ps.make_shape(32, 8, 128)
+    csv = tmp_path / "t.csv"
+    plain = ps.ps_profile_grid(sh, (256,), (32,), (1024,), 2, 2, 5, 3000)
+    both = ps.ps_profile_grid(sh, (256,), (32,), (1024,), 2, 2, 5, 3000, str(csv), include_kv_write=True)
+    assert [(r.seed, r.kv_tokens, r.token_batch) for r in plain] == [(r.seed, r.kv_tokens, r.token_batch) for r in both]
+    assert all(0 < r.latency_us < 1e5 for r in both)
+    # the append adds a kernel launch to every run: it cannot make the step much faster
+    assert np.median([r.latency_us for r in both]) > 0.8 * np.median([r.latency_us for r in plain])
+    assert csv.read_text().splitlines()[1].startswith("attn+kv_write,256,32,1024")
+
+
 def test_grid_rejects_bad_specs():
     sh = ps.make_shape(32, 8, 128)
     for args in [((), (8,), (512,), 1, 1, 1), ((64,), (8,), (1,), 1, 1, 1), ((64,), (8,), (512,), 0, 1, 1), ((0,), (0,), (512,), 1, 1, 1)]:

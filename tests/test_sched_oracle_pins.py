@@ -177,6 +177,21 @@ def test_table_lookup_interpolates_in_batch_and_clamps():
     assert so.table_predict(lines, 200, 1000, 4e9) == pytest.approx(0.5 * (11.0 + 56.0))
 
 
+def test_batch_term_and_scaling():
+    lines = [(100, 10.0, 1e-3, 1e-9), (200, 20.0, 2e-3, 2e-9), (900, 50.0, 3e-3, 0.0)]
+    # GEMM(B) sampled at 64, 128 and 512 tokens: 100 -> 30 + 36/64 * 20 = 41.25, 200 -> 50 + 72/384 * 100, 900 -> clamped
+    got = so.table_add_batch_term(lines, [(512, 150.0), (64, 30.0), (128, 50.0)])
+    assert [ln[0] for ln in got] == [100, 200, 900]
+    assert got[0][1] == pytest.approx(10.0 + 41.25) and got[1][1] == pytest.approx(20.0 + 50.0 + 72.0 / 384.0 * 100.0)
+    assert got[2][1] == pytest.approx(50.0 + 150.0)
+    assert [ln[2:] for ln in got] == [ln[2:] for ln in lines]          # the slopes are untouched
+    assert so.table_add_batch_term(lines, [(300, 7.0)])[0][1] == pytest.approx(17.0)  # one sample: a constant
+    # a sum of per-layer terms over 32 layers is 32 times every coefficient, hence 32 times every prediction
+    x32 = so.table_scale(lines, 32.0)
+    for b, kv, pf in [(100, 5000, 0.0), (150, 123456, 3e9), (5000, 10, 1e12)]:
+        assert so.table_predict(x32, b, kv, pf) == pytest.approx(32.0 * so.table_predict(lines, b, kv, pf))
+
+
 def test_admission_uses_the_peak_and_the_current_batch_size():
     # table(b, kv) = 2 b + 0.01 kv
     lines = [(1, 2.0, 0.01, 1e-9), (1001, 2002.0, 0.01, 1e-9)]

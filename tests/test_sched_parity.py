@@ -86,6 +86,28 @@ def test_table_build_and_predict_match_the_oracle():
             S.ps_table_free(t)
 
 
+def test_batch_term_and_scale_match_the_oracle():
+    rng = np.random.default_rng(26)
+    lines = [(72, 14.0, 2.2e-4, 0.0), (96, 16.0, 2.4e-4, 6e-10), (320, 30.0, 2.5e-4, 1.0e-9), (2304, 60.0, 2.7e-4, 1.0e-9)]
+    for samples in ([(64, 30.0), (128, 50.0), (512, 150.0), (4096, 900.0)], [(300, 7.0)], [(2304, 1.0), (72, 2.0)]):
+        t = S.ps_table_from_lines(*zip(*lines))
+        try:
+            perm = rng.permutation(len(samples))
+            S.ps_table_add_batch_term(t, [samples[i][0] for i in perm], [samples[i][1] for i in perm])
+            S.ps_table_scale(t, 32.0)
+            want = so.table_scale(so.table_add_batch_term(lines, samples), 32.0)
+            got = list(zip(*[x.tolist() for x in S.ps_table_get_lines(t)]))
+            assert len(got) == len(want)
+            for g, w in zip(got, want):
+                assert g[0] == w[0] and all(close(a, b) for a, b in zip(g[1:], w[1:]))
+            with pytest.raises(ps.PsError):
+                S.ps_table_add_batch_term(t, [8, 8], [1.0, 2.0])
+            with pytest.raises(ps.PsError):
+                S.ps_table_scale(t, 0.0)
+        finally:
+            S.ps_table_free(t)
+
+
 def test_table_rejects_bad_input():
     with pytest.raises(ps.PsError):
         S.ps_table_from_lines([10, 10], [1.0, 2.0], [0.1, 0.1])  # duplicate batch size
