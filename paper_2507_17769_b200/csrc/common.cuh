@@ -8,6 +8,8 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <mutex>
+
 #include "../../include/polyserve_attn.h"
 
 namespace ps {
@@ -27,6 +29,25 @@ void clear_error();
     } while (0)
 
 ps_status check_shape(const ps_shape* s);
+
+// Kernel attributes (the opt-in to large dynamic shared memory) belong to a device: run `configure` once
+// per device the calling process launches on.  `state` is a function-local static of the caller.
+struct PerDeviceOnce {
+    std::mutex mu;
+    uint64_t done[4] = {0, 0, 0, 0};  // one bit per device ordinal (up to 256)
+};
+template <typename F>
+ps_status once_per_device(PerDeviceOnce& state, F configure) {
+    int dev = 0;
+    PS_CUDA_TRY(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(state.mu);
+    uint64_t& word = state.done[(dev >> 6) & 3];
+    const uint64_t bit = 1ull << (dev & 63);
+    if (word & bit) return PS_OK;
+    const ps_status st = configure();
+    if (st == PS_OK) word |= bit;
+    return st;
+}
 
 // ---------------------------------------------------------------------------
 // KV pool layout

@@ -167,7 +167,6 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
     auto combine = [&](int midx, int qtok, int g) {
         __syncwarp();  // lane 0's acquiring increment is ordered before every lane's partial loads
         const DecodeMerge dm = p.dmerge[midx];
-        constexpr int V = D / 32;  // floats per lane
         // The n_seg * G log-sum-exps are contiguous (segment-major, head-minor).  Lane i reads entries
         // i, i + 32, ...; since G divides 32 they all belong to head i % G, so the per-head max and
         // sum are reductions over the lanes that are congruent mod G.
@@ -440,11 +439,12 @@ int decode_warps_per_sm() { return kWarps; }
 template <int D>
 static ps_status launch_decode_d(const RunArgs& a) {
     using Cfg = DecodeCfg<D>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    const ps_status cfg = once_per_device(configured, []() -> ps_status {
         PS_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-        configured = true;
-    }
+        return PS_OK;
+    });
+    if (cfg != PS_OK) return cfg;
     DecodeParams p;
     p.pool = a.pool;
     p.num_pages = a.num_pages;

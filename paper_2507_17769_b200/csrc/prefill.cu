@@ -769,11 +769,12 @@ EncodeTiledFn tensor_map_encoder() {
 template <int D>
 static ps_status launch_prefill_d(const RunArgs& a) {
     using Cfg = PrefillCfg<D>;
-    static bool configured = false;
-    if (!configured) {
+    static PerDeviceOnce configured;
+    const ps_status cfg = once_per_device(configured, []() -> ps_status {
         PS_CUDA_TRY(cudaFuncSetAttribute(prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
-        configured = true;
-    }
+        return PS_OK;
+    });
+    if (cfg != PS_OK) return cfg;
     PrefillParams p;
     p.pool = a.pool;
     p.num_pages = a.num_pages;
