@@ -10,7 +10,10 @@ and merge kernels).  The default workload is the decode-only 8B-class batch
 L2); the headline value is the KV bytes the decode rows must stream divided by
 the step time.  With N > 1 (torchrun) every rank runs its own batch of the same
 law (weak scaling, no data-path collective); the step time is the maximum over
-ranks and the value the sum of all ranks' bytes over that time.
+ranks and the value the sum of all ranks' bytes over that time.  With
+``--shard heads`` the ranks instead split ONE batch by KV head (rank k takes kv
+heads [k Hkv / N, (k + 1) Hkv / N) and their q heads; attention needs no
+exchange between heads), which is strong scaling.
 
 Prints one JSON line.  ``--impl reference`` times the CPU oracle instead.
 """
@@ -130,6 +133,20 @@ def reduce_over_ranks(local_ms: float, local_units: float, world: int, device=No
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     dist.all_reduce(u, op=dist.ReduceOp.SUM)
     return float(t.item()), float(u.item())
+
+
+def shard_batch(make, seed, rank, world, shard):
+    """This rank's share of the job.  "requests": its own batch of the same law (replicas, weak scaling).  "heads":
+    the one batch of `seed`, cut by KV head -- same lengths and pages on every rank, Hkv / world kv heads and
+    their q heads each (strong scaling; head slices never exchange anything inside attention)."""
+    if shard == "requests" or world == 1:
+        return make(seed + 100 * rank)
+    full = make(seed)
+    s = full.shape
+    if s.n_kv_heads % world != 0:
+        raise SystemExit("--shard heads: %d kv heads do not divide over %d ranks" % (s.n_kv_heads, world))
+    part = gen.Shape(s.n_q_heads // world, s.n_kv_heads // world, s.head_dim, s.page_size)
+    return gen.make_batch(part, seed, full.prior, full.q_len)
 
 
 def oracle_sample(batch, budget_flops=6e10):
@@ -263,7 +280,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
 
     desc, make, seed = WORKLOADS[args.workload]
-    batch = make(seed + 100 * rank)  # each rank its own batch of the same law
+    batch = shard_batch(make, seed, rank, world, args.shard)
     s = batch.shape
     db = DeviceBatch(batch, poison=False, device=dev)
     pa = db.pa
@@ -372,12 +389,13 @@ def run_ours(args):
             extra.update(components_alone(pa, batch, db, out, args.steps, peaks))
         line = {
             "metric": METRIC, "value": value, "unit": "TB/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
-            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-            "data": "synthetic",
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "strong" if args.shard == "heads" and world > 1 else "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": desc, "kv_bytes_per_step_per_gpu": dec_bytes, "prefill_flops_per_step_per_gpu": pf_flops,
                        "l2": "inputs larger than L2 (%.0f MB of KV per step), no flush" % (dec_bytes / 1e6),
                        "decode_items": info.n_decode_items, "prefill_items": info.n_prefill_items,
-                       "merge_rows": info.n_merge_rows, "parallelism": "replicas x%d" % world},
+                       "merge_rows": info.n_merge_rows,
+                       "parallelism": ("kv heads x%d" if args.shard == "heads" and world > 1 else "replicas x%d") % world},
             "clocks": clocks.summary(),
             "e2e": {"value": e2e_units / (e2e_ms * 1e-3) / 1e12, "unit": "TB/s", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -411,6 +429,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=1, choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--shard", default="requests", choices=["requests", "heads"],
+                    help="what N > 1 ranks split: requests (each rank its own batch; default) or the KV heads of one batch")
     args = ap.parse_args()
     if args.impl == "reference":
         args.steps = min(args.steps, 5)  # each step is seconds of CPU work

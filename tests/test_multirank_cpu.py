@@ -35,6 +35,13 @@ def _rank_main(rank, world, port, out):
     ps.ps_plan_free(plan)
     local_ms = 1.0 + rank  # stand-in for the device time
     ms, units = bench.reduce_over_ranks(local_ms, float(batch.decode_bytes()), world)
+    # the other way to split the job: one batch, cut by KV head -- same lengths on every rank, half the heads each
+    full = gen.config1(1001)
+    part = bench.shard_batch(gen.config1, 1001, rank, world, "heads")
+    assert (part.shape.n_q_heads, part.shape.n_kv_heads) == (16, 4) and (part.prior == full.prior).all()
+    assert (part.block_table == full.block_table).all()
+    _, head_units = bench.reduce_over_ranks(local_ms, float(part.decode_bytes()), world)
+    assert head_units == float(full.decode_bytes())  # the shards' bytes add up to the whole batch's
     out.put((rank, ms, units, float(batch.decode_bytes()), info.n_decode_items))
     dist.barrier()
     dist.destroy_process_group()
