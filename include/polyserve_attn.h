@@ -191,9 +191,10 @@ ps_status ps_plan_get_items(const ps_plan *plan, int32_t *decode_items_out, int6
  * `stream` with events, into one of two slots of the workspace so that it can
  * run under the previous run's kernels), then the prefill, decode and merge
  * kernels run; for a batch with both row classes the decode kernel may run on
- * a second stream of the plan, beside the prefill kernel on disjoint SMs, and
- * is joined back into `stream` before the call's work is complete in stream
- * order.  Consecutive runs of one plan must be issued to the
+ * a second stream of the plan, beside the prefill kernel on disjoint SMs (the
+ * merge kernel then follows the prefill kernel at once, under the decode
+ * kernel), and is joined back into `stream` before the call's work is
+ * complete in stream order.  Consecutive runs of one plan must be issued to the
  * same stream, or be ordered by the caller: they share the partial buffers.
  * Returns host-detectable errors only (PS_ERR_INVALID, PS_ERR_WORKSPACE,
  * PS_ERR_CUDA); errors seen on the device are read with ps_plan_status.

@@ -594,6 +594,7 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     const bool rec = pl->timing && (size_t)(pl->timed_runs + 1) * 6 <= pl->tev.size();
     cudaEvent_t* ev = rec ? &pl->tev[(size_t)pl->timed_runs * 6] : nullptr;
     ps_status st = PS_OK;
+    bool merged = false;  // the merge kernel has been launched already
     if (pl->concurrent && pl->side_stream) {
         // Mixed batch: the decode kernel runs on its share of the SMs on a second stream while the
         // prefill kernel runs on the rest.  Both need about 200 KB of shared memory per CTA, so each SM
@@ -611,6 +612,15 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
         st = launch_prefill(a);
         if (st != PS_OK) return st;
         if (rec) cudaEventRecord(ev[1], s);
+        if (!(a.w.n_prefill_ctas == 0 && a.w.n_prefill > a.pf_sms)) {
+            // Only this launch writes prefill partials: combine them right behind it, on the SMs it leaves, while
+            // the decode kernel is still streaming (decode rows are combined inside the decode kernel).
+            if (rec) cudaEventRecord(ev[4], s);
+            st = launch_merge(a);
+            if (st != PS_OK) return st;
+            if (rec) cudaEventRecord(ev[5], s);
+            merged = true;
+        }
         if (a.w.n_prefill_ctas == 0 && a.w.n_prefill > a.pf_sms) {
             // dynamic item queue: once the decode CTAs have left their SMs, as many more prefill CTAs
             // start there and help drain the same queue
@@ -632,12 +642,12 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
         if (st != PS_OK) return st;
         if (rec) cudaEventRecord(ev[3], s);
     }
-    if (rec) cudaEventRecord(ev[4], s);
-    st = launch_merge(a);
-    if (rec) {
-        cudaEventRecord(ev[5], s);
-        ++pl->timed_runs;
+    if (!merged) {
+        if (rec) cudaEventRecord(ev[4], s);
+        st = launch_merge(a);
+        if (rec) cudaEventRecord(ev[5], s);
     }
+    if (rec) ++pl->timed_runs;
     if (pl->copy_stream && st == PS_OK) {
         PS_CUDA_TRY(cudaEventRecord(pl->ev_done[slot], s));
         pl->done_valid[slot] = true;
