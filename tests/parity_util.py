@@ -46,15 +46,28 @@ def oracle_subset(batch, reqs, rows=None):
     return out, lse, np.asarray(packed)
 
 
-def compare(gpu_out, gpu_lse, want_out, want_lse, packed=None, what=""):
-    """gpu_out: torch bf16 [T, Hq, d] (device), gpu_lse: torch fp32 [T, Hq] or None."""
+def compare(gpu_out, gpu_lse, want_out, want_lse, packed=None, what="", few_key_rows=False):
+    """gpu_out: torch bf16 [T, Hq, d] (device), gpu_lse: torch fp32 [T, Hq] or None.
+
+    ``few_key_rows``: for batches made mostly of rows that see one or two keys.  Such a row's output is as
+    large as a single V value (up to 4 and more for N(0,1) data), and a bf16 result cannot be closer to the exact
+    one than half a unit in its last place, |x| 2^-8 at worst: 0.016 at |x| = 4.1 however the kernel computes.
+    The bounds then scale with the values: per element max(1e-2, |want| 2^-7) (the output's own rounding plus as
+    much again for the bf16-rounded weights), and for the mean max(1e-3, mean|want| 2^-8).  Batches shaped like
+    the target's configs average over many keys and are held to the plain 1e-2 / 1e-3."""
     got = gpu_out.float().cpu().numpy().astype(np.float64)
     if packed is not None:
         got = got[packed]
     assert np.all(np.isfinite(got)), "%s: non-finite output" % what
     err = np.abs(got - want_out)
-    assert err.max() <= MAX_ABS, "%s: max-abs %.3e" % (what, err.max())
-    assert err.mean() <= MEAN_ABS, "%s: mean-abs %.3e" % (what, err.mean())
+    if few_key_rows:
+        bound = np.maximum(MAX_ABS, np.abs(want_out) * 2.0 ** -7)
+        worst = np.unravel_index(np.argmax(err - bound), err.shape)
+        assert np.all(err <= bound), "%s: error %.3e at a value of %.4f" % (what, err[worst], want_out[worst])
+        assert err.mean() <= max(MEAN_ABS, np.abs(want_out).mean() * 2.0 ** -8), "%s: mean-abs %.3e" % (what, err.mean())
+    else:
+        assert err.max() <= MAX_ABS, "%s: max-abs %.3e" % (what, err.max())
+        assert err.mean() <= MEAN_ABS, "%s: mean-abs %.3e" % (what, err.mean())
     if gpu_lse is not None:
         gl = gpu_lse.cpu().numpy().astype(np.float64)
         if packed is not None:

@@ -1,6 +1,8 @@
 """Randomised mixed batches against the oracle: shapes, row mix, lengths, planner segment sizes and SM counts drawn
-from a seeded generator, pools poisoned with NaN.  Same tolerance as the other parity tests (max-abs <= 1e-2,
-mean-abs <= 1e-3 on bf16 outputs, lse to 2e-3); every case also runs twice and must repeat bit for bit."""
+from a seeded generator, pools poisoned with NaN.  Tolerance: that of the other parity tests (max-abs <= 1e-2,
+mean-abs <= 1e-3 on bf16 outputs, lse to 2e-3), widened in proportion to the value where a bf16 output cannot do
+better (rows that see one or two keys are as large as single V values; see parity_util.compare); every case also
+runs twice and must repeat bit for bit."""
 import os
 
 import numpy as np
@@ -37,7 +39,7 @@ def draw_batch(rng, case):
     return gen.make_batch(shape, 4000 + case, [prior[i] for i in order], [q_len[i] for i in order])
 
 
-@pytest.mark.parametrize("case", range(int(os.environ.get("PS_FUZZ_CASES", "18"))))  # more cases: PS_FUZZ_CASES=300
+@pytest.mark.parametrize("case", range(int(os.environ.get("PS_FUZZ_CASES", "40"))))  # more cases: PS_FUZZ_CASES=300
 def test_random_mixed_batch(case):
     import torch
 
@@ -53,7 +55,7 @@ def test_random_mixed_batch(case):
     out, lse = db.run()
     db.pa.check()
     want, want_lse, _ = oracle_subset(batch, range(batch.n))
-    compare(out, lse, want, want_lse, what="fuzz case %d" % case)
+    compare(out, lse, want, want_lse, what="fuzz case %d" % case, few_key_rows=True)
     out2, lse2 = db.run()
     db.pa.check()
     assert torch.equal(out.view(torch.int16), out2.view(torch.int16)) and torch.equal(lse, lse2)
