@@ -190,15 +190,30 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
             float4 acc[NV];
 #pragma unroll
             for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 2
-            for (int s = 0; s < dm.n_seg; ++s) {  // fixed segment order
-                const int64_t slot = (int64_t)dm.base + s * p.G + hh;
-                const float w = __expf(__ldcg(p.part_lse + slot) - M);
-                const float4* po = reinterpret_cast<const float4*>(p.part_o + slot * D) + part * NV;
+            // fixed segment order; kAhead segments' rows are requested before the first is used, so that a long
+            // list of segments costs about one trip to L2 per kAhead of them
+            constexpr int kAhead = NV <= 2 ? 8 : NV <= 4 ? 4 : 2;  // at most 16 float4 in flight per lane
+            for (int s0 = 0; s0 < dm.n_seg; s0 += kAhead) {
+                float4 x[kAhead][NV];
+                float lw[kAhead];
 #pragma unroll
-                for (int v = 0; v < NV; ++v) {
-                    const float4 x = __ldcg(po + v);
-                    acc[v].x += w * x.x; acc[v].y += w * x.y; acc[v].z += w * x.z; acc[v].w += w * x.w;
+                for (int k = 0; k < kAhead; ++k) {
+                    const int sk = min(s0 + k, dm.n_seg - 1);  // past the end: a repeat that is not accumulated
+                    const int64_t slot = (int64_t)dm.base + sk * p.G + hh;
+                    lw[k] = __ldcg(p.part_lse + slot);
+                    const float4* po = reinterpret_cast<const float4*>(p.part_o + slot * D) + part * NV;
+#pragma unroll
+                    for (int v = 0; v < NV; ++v) x[k][v] = __ldcg(po + v);
+                }
+#pragma unroll
+                for (int k = 0; k < kAhead; ++k) {
+                    if (s0 + k < dm.n_seg) {  // warp-uniform
+                        const float w = __expf(lw[k] - M);
+#pragma unroll
+                        for (int v = 0; v < NV; ++v) {
+                            acc[v].x += w * x[k][v].x; acc[v].y += w * x[k][v].y; acc[v].z += w * x[k][v].z; acc[v].w += w * x[k][v].w;
+                        }
+                    }
                 }
             }
             uint2* op = reinterpret_cast<uint2*>(p.out + orow * D) + part * NV;

@@ -17,7 +17,11 @@ namespace ps {
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 constexpr int kDecodeUnitsPerWarp = 1;  // work units per resident warp (measured: 1 beats 2 and 3 on the decode-only batch)
-constexpr int kDecodeMinPages = 8;      // smallest decode unit (pages)
+// Smallest decode unit (pages) of a batch too small to give every warp its share: between 4 and 8, so that the
+// longest row is cut into about 16 pieces at most.  Finer cuts spread a small batch over more warps (64 rows of
+// 64 tokens: 13 us instead of 20; 8 rows of 512: 16 instead of 23), but every further piece of a row is one more
+// partial result for the one warp that combines them (one row of 4096 tokens: 22 us at 32 pieces, 26 at 64).
+constexpr int kDecodeMinPagesLo = 4, kDecodeMinPagesHi = 8, kDecodePiecesPerRow = 16;
 constexpr int kPrefillKeyTile = 128;    // keys per tensor-core tile
 // Measured on B200 (decode: bandwidth against the number of SMs the kernel runs on; prefill: time of one
 // key-tile step of a q tile pair), used to split the SMs of a mixed batch between the two kernels.
@@ -85,16 +89,21 @@ static int query_num_sms() {
 static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len, const std::vector<int32_t>& q_start,
                         const ps_plan_opts* opts, int64_t* n_slots) {
     const int Hkv = pl->shape.n_kv_heads, G = pl->shape.n_q_heads / Hkv;
-    int64_t total_pages = 0;
+    int64_t total_pages = 0, longest = 0;
     for (int r = 0; r < pl->n; ++r)
-        if (q_len[r] == 1) total_pages += (int64_t)((prior[r] + 1 + kPage - 1) / kPage) * Hkv;
+        if (q_len[r] == 1) {
+            const int64_t pages = (prior[r] + 1 + kPage - 1) / kPage;
+            total_pages += pages * Hkv;
+            longest = std::max(longest, pages);
+        }
     if (total_pages == 0) return;
+    const int64_t min_pages = std::min<int64_t>(kDecodeMinPagesHi, std::max<int64_t>(kDecodeMinPagesLo, (longest + kDecodePiecesPerRow - 1) / kDecodePiecesPerRow));
     int64_t per_unit;
     if (opts && opts->decode_segment_tokens > 0) {
         per_unit = std::max(1, opts->decode_segment_tokens / kPage);
     } else {
         const int64_t target = (int64_t)pl->dec_sms * decode_warps_per_sm() * kDecodeUnitsPerWarp;
-        per_unit = std::max<int64_t>(kDecodeMinPages, (total_pages + target - 1) / target);
+        per_unit = std::max<int64_t>(min_pages, (total_pages + target - 1) / target);
     }
     pl->info.decode_segment_tokens = (int32_t)(per_unit * kPage);
 
