@@ -28,6 +28,7 @@ constexpr int kPrefillKeyTile = 128;    // keys per tensor-core tile
 constexpr double kDecodePeakBytesPerSec = 6.7e12;
 constexpr double kDecodeSharedPeakBytesPerSec = 6.0e12;  // decode rows beside a running prefill kernel
 constexpr double kDecodeBytesPerSecPerSm = 115e9;
+constexpr double kDecodeAloneBytesPerSecPerSm = 135e9;  // per SM with the memory system to itself
 constexpr double kPrefillStepSec = 2.5e-6;
 constexpr double kKernelFloorSec = 12e-6;
 
@@ -387,6 +388,16 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
                 if (std::max(t_dec(nd), t_pf(nd)) <= 1.015 * best_t && t_pf(nd) <= 0.8 * t_dec(nd)) hi = nd;
             best_n = (best_n + hi) / 2 / 4 * 4;
             const double t_seq = dec_bytes / kDecodePeakBytesPerSec + pf_steps * kPrefillStepSec / pl->num_sms + 2 * kKernelFloorSec;
+            // The decode rows pay the shared rate only while the prefill kernel runs; once it has ended they stream
+            // at the rate their CTAs reach alone.  A short chunk beside many decode rows is therefore cheaper than
+            // the model above says, which matters for the choice against running the two one after the other.
+            if (best_n > 0) {
+                const double pf_work = pf_steps * kPrefillStepSec / (pl->num_sms - best_n);
+                const double shared = std::min(kDecodeSharedPeakBytesPerSec, best_n * kDecodeBytesPerSecPerSm);
+                const double alone = std::min(kDecodePeakBytesPerSec, best_n * kDecodeAloneBytesPerSecPerSm);
+                const double dec_work = dec_bytes <= shared * pf_work ? dec_bytes / shared : pf_work + (dec_bytes - shared * pf_work) / alone;
+                best_t = std::min(best_t, std::max(pf_work, dec_work) + kKernelFloorSec);
+            }
             if (best_n > 0 && best_t < 0.95 * t_seq) {
                 pl->dec_sms = best_n;
                 pl->pf_sms = pl->num_sms - best_n;
