@@ -157,6 +157,8 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
 // (fitted to per-CTA run times on B200: 2.2 us per step, about 3 us per item, 1.2 us more for a masked tile)
 constexpr double kPrefillFixedCost = 1.5;
 constexpr double kPrefillMaskedExtra = 0.5;  // the diagonal tile of an item takes the slower masked softmax
+constexpr double kPrefillCutCost = 3.0;
+constexpr double kPrefillWholeItemSlack = 1.12;  // uncut items are taken if the busiest CTA stays within this of an even split
 constexpr double kPrefillMinCtaCost = 4.0;  // do not spread the work thinner than this per CTA (two key tiles)
 
 static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len, const std::vector<int32_t>& q_start,
@@ -183,7 +185,7 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
     // cut[i] = key-tile indices at which tile i is cut into pieces (ascending, exclusive of 0 and key_tiles)
     std::vector<std::vector<int>> cuts(tiles.size());
     // owner CTA of the first piece of each tile and of each following piece, for the static partition
-    bool static_partition = false;
+    bool static_partition = false, whole_items = false;
     if (opts && opts->prefill_segment_tokens > 0) {
         const int seg_tiles = std::max(1, opts->prefill_segment_tokens / kPrefillKeyTile);
         pl->info.prefill_segment_tokens = seg_tiles * kPrefillKeyTile;
@@ -203,6 +205,39 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
         double total = 0;
         for (const Tile& t : tiles) total += kPrefillFixedCost + t.key_tiles + kPrefillMaskedExtra;
         const int n_cta = (int)std::max<double>(1, std::min<double>(pl->pf_sms, total / kPrefillMinCtaCost));
+        // Many short items (fresh prompts): whole items, longest first, each to the CTA with the least work so far.
+        // If that comes within kPrefillWholeItemSlack of an even split, nothing is cut: no partial rows, no merge
+        // kernel, no item paying its fixed cost twice.
+        if ((int)tiles.size() >= n_cta) {
+            std::vector<int> order(tiles.size());
+            for (size_t i = 0; i < tiles.size(); ++i) order[i] = (int)i;
+            std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return tiles[a].key_tiles > tiles[b].key_tiles; });
+            std::vector<double> load(n_cta, 0.0);
+            std::vector<int> owner(tiles.size());
+            // a heap would do; CTAs are at most 148 and items a few hundred
+            for (int i : order) {
+                int best = 0;
+                for (int c = 1; c < n_cta; ++c)
+                    if (load[c] < load[best]) best = c;
+                owner[i] = best;
+                load[best] += kPrefillFixedCost + tiles[i].key_tiles + kPrefillMaskedExtra;
+            }
+            const double makespan = *std::max_element(load.begin(), load.end());
+            // (cutting is not free either: the merge kernel and the partial rows cost about kPrefillCutCost steps)
+            if (makespan <= std::max(kPrefillWholeItemSlack * total / n_cta, total / n_cta + kPrefillCutCost)) {
+                std::vector<Tile> sorted;
+                sorted.reserve(tiles.size());
+                pl->prefill_cta_start.assign(1, 0);
+                for (int c = 0; c < n_cta; ++c) {
+                    for (int i : order)
+                        if (owner[i] == c) sorted.push_back(tiles[i]);
+                    pl->prefill_cta_start.push_back((int32_t)sorted.size());
+                }
+                tiles.swap(sorted);
+                whole_items = true;
+            }
+        }
+        if (!whole_items) {
         // CTA k ends where the running cost passes (k + 1) * quota (absolute marks, so rounding does not pile
         // up).  A share that ends inside an item makes the rest of that item pay the fixed cost again, and how
         // many shares do depends on the quota itself: bisect for the smallest quota that does not leave the
@@ -249,6 +284,7 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
         }
         while ((int)pl->prefill_cta_start.size() < n_cta) pl->prefill_cta_start.push_back(n_items);  // CTAs left without work
         pl->prefill_cta_start.push_back(n_items);
+        }
     }
 
     for (size_t i = 0; i < tiles.size(); ++i) {
