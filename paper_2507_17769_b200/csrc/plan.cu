@@ -208,7 +208,7 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
         // Many short items (fresh prompts): whole items, longest first, each to the CTA with the least work so far.
         // If that comes within kPrefillWholeItemSlack of an even split, nothing is cut: no partial rows, no merge
         // kernel, no item paying its fixed cost twice.
-        if ((int)tiles.size() >= n_cta) {
+        {
             std::vector<int> order(tiles.size());
             for (size_t i = 0; i < tiles.size(); ++i) order[i] = (int)i;
             std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return tiles[a].key_tiles > tiles[b].key_tiles; });
