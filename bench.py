@@ -368,23 +368,34 @@ def run_ours(args):
         k, v = gen_cuda.gen_kv(batch.seed, r, int(batch.prior[r]), int(batch.kv_len[r]), s.n_kv_heads, s.head_dim, dev)
         new_k.append(k)
         new_v.append(v)
-    h_q = db.q.cpu().pin_memory()
-    h_k = torch.cat(new_k).cpu().pin_memory()
-    h_v = torch.cat(new_v).cpu().pin_memory()
-    h_bt = torch.from_numpy(batch.block_table).pin_memory()
+    # one pinned staging buffer and one device buffer hold the step's inputs back to back (Q | K | V | block table,
+    # each 256-byte aligned), so that a step's inputs cross in a single copy
+    parts = [db.q.cpu().contiguous().view(torch.uint8).reshape(-1), torch.cat(new_k).cpu().contiguous().view(torch.uint8).reshape(-1),
+             torch.cat(new_v).cpu().contiguous().view(torch.uint8).reshape(-1),
+             torch.from_numpy(batch.block_table).contiguous().view(torch.uint8).reshape(-1)]
+    offs, total = [], 0
+    for t in parts:
+        offs.append(total)
+        total += (t.numel() + 255) // 256 * 256
+    h_in = torch.zeros(total, dtype=torch.uint8).pin_memory()
+    for t, o in zip(parts, offs):
+        h_in[o : o + t.numel()] = t
+    d_in = torch.empty(total, dtype=torch.uint8, device=dev)
+
+    def view(i, dtype, shape):
+        return d_in[offs[i] : offs[i] + parts[i].numel()].view(dtype).reshape(shape)
+
+    n_new = int(batch.q_len.sum())
+    d_q = view(0, torch.bfloat16, db.q.shape)
+    d_k = view(1, torch.bfloat16, (n_new, s.n_kv_heads, s.head_dim))
+    d_v = view(2, torch.bfloat16, (n_new, s.n_kv_heads, s.head_dim))
+    d_bt = view(3, torch.int32, db.block_table.shape)
     h_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
-    d_q = torch.empty_like(db.q)
-    d_k = torch.empty(h_k.shape, dtype=h_k.dtype, device=dev)
-    d_v = torch.empty(h_v.shape, dtype=h_v.dtype, device=dev)
-    d_bt = torch.empty_like(db.block_table)
-    h2d = h_q.numel() * 2 + h_k.numel() * 2 + h_v.numel() * 2 + h_bt.numel() * 4
+    h2d = sum(t.numel() for t in parts)
     d2h = h_out.numel() * 2
 
     def e2e_step():
-        d_q.copy_(h_q, non_blocking=True)
-        d_k.copy_(h_k, non_blocking=True)
-        d_v.copy_(h_v, non_blocking=True)
-        d_bt.copy_(h_bt, non_blocking=True)
+        d_in.copy_(h_in, non_blocking=True)
         pa.write(d_k, d_v, d_bt, batch.prior, batch.q_len, max_pages=batch.max_pages)
         pa.plan(batch.prior, batch.q_len, batch.max_pages)
         pa.run(d_q, d_bt, out=out, want_lse=False)
