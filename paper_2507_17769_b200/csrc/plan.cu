@@ -7,7 +7,9 @@
 #include <cstdlib>
 #include <cmath>
 #include <cstring>
+#include <functional>
 #include <new>
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -97,7 +99,12 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
             total_pages += pages * Hkv;
             longest = std::max(longest, pages);
         }
-    if (total_pages == 0) return;
+    if (total_pages == 0) {
+        pl->pieces.clear();
+        pl->units.clear();
+        pl->dmerge.clear();
+        return;
+    }
     const int64_t min_pages = std::min<int64_t>(kDecodeMinPagesHi, std::max<int64_t>(kDecodeMinPagesLo, (longest + kDecodePiecesPerRow - 1) / kDecodePiecesPerRow));
     int64_t per_unit;
     if (opts && opts->decode_segment_tokens > 0) {
@@ -108,48 +115,66 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
     }
     pl->info.decode_segment_tokens = (int32_t)(per_unit * kPage);
 
+    // Upper bounds on the counts (a piece ends where its row or its unit ends), so that the lists are filled
+    // in place and trimmed once.
+    int64_t n_rows = 0;
+    for (int r = 0; r < pl->n; ++r) n_rows += q_len[r] == 1 ? Hkv : 0;
+    const size_t max_units = (size_t)((total_pages + per_unit - 1) / per_unit);
+    pl->pieces.resize((size_t)n_rows + max_units);
+    pl->units.resize(max_units);
+    pl->dmerge.resize(std::min<size_t>((size_t)n_rows, max_units));
+    DecodePiece* const pieces = pl->pieces.data();
+    DecodeUnit* const units = pl->units.data();
+    DecodeMerge* const dmerge = pl->dmerge.data();
+    int32_t n_pieces = 0, n_units = 0, n_dmerge = 0;
+    int64_t slots = *n_slots;
     int64_t room = 0;  // pages the open unit can still take
     for (int r = 0; r < pl->n; ++r) {
         if (q_len[r] != 1) continue;
         const int kv_len = prior[r] + 1;
         const int pages = (kv_len + kPage - 1) / kPage;
+        const int32_t q_tok = q_start[r];
         for (int g = 0; g < Hkv; ++g) {
-            const size_t first_piece = pl->pieces.size();
+            const int32_t first_piece = n_pieces;
             int pg = 0;
             while (pg < pages) {
                 if (room == 0) {
-                    pl->units.push_back(DecodeUnit{(int32_t)pl->pieces.size(), (int32_t)pl->pieces.size()});
+                    if (n_units > 0) units[n_units - 1].piece_end = n_pieces;
+                    units[n_units++].piece_begin = n_pieces;
                     room = per_unit;
                 }
                 const int take = (int)std::min<int64_t>(room, pages - pg);
-                DecodePiece pc{};
+                DecodePiece& pc = pieces[n_pieces++];
                 pc.req = r;
                 pc.kv_head = g;
                 pc.page_begin = pg;
                 pc.page_end = pg + take;
-                pc.q_tok = q_start[r];
+                pc.q_tok = q_tok;
                 pc.part_slot = -1;
                 pc.kv_len = kv_len;
-                pl->pieces.push_back(pc);
-                pl->units.back().piece_end = (int32_t)pl->pieces.size();
+                pc.merge_idx = 0;
                 pg += take;
                 room -= take;
             }
-            const size_t cnt = pl->pieces.size() - first_piece;
+            const int32_t cnt = n_pieces - first_piece;
             if (cnt > 1) {
-                DecodeMerge dm{};
-                dm.base = (int32_t)*n_slots;
-                dm.n_seg = (int32_t)cnt;
-                for (size_t s = 0; s < cnt; ++s) {
-                    pl->pieces[first_piece + s].part_slot = (int32_t)(*n_slots + (int64_t)s * G);
-                    pl->pieces[first_piece + s].merge_idx = (int32_t)pl->dmerge.size();
+                for (int32_t s = 0; s < cnt; ++s) {
+                    pieces[first_piece + s].part_slot = (int32_t)(slots + (int64_t)s * G);
+                    pieces[first_piece + s].merge_idx = n_dmerge;
                 }
-                pl->dmerge.push_back(dm);
-                pl->decode_merge_rows += G;
-                *n_slots += (int64_t)cnt * G;
+                dmerge[n_dmerge].base = (int32_t)slots;
+                dmerge[n_dmerge].n_seg = cnt;
+                ++n_dmerge;
+                slots += (int64_t)cnt * G;
             }
         }
     }
+    if (n_units > 0) units[n_units - 1].piece_end = n_pieces;
+    pl->pieces.resize((size_t)n_pieces);
+    pl->units.resize((size_t)n_units);
+    pl->dmerge.resize((size_t)n_dmerge);
+    pl->decode_merge_rows += (int64_t)n_dmerge * G;
+    *n_slots = slots;
 }
 
 // Cost model of the prefill kernel in units of one 128-key tile step: an item pays a fixed
@@ -167,6 +192,10 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
     const int tile_tok = kPrefillRowsPerItem / G;
     struct Tile { int r, g, tok0, n_tok, first_pos, key_tiles; };
     std::vector<Tile> tiles;
+    size_t n_tiles = 0;
+    for (int r = 0; r < pl->n; ++r)
+        if (q_len[r] > 1) n_tiles += (size_t)((q_len[r] + tile_tok - 1) / tile_tok) * Hkv;
+    tiles.reserve(n_tiles);
     int64_t total_key_tiles = 0;
     for (int r = 0; r < pl->n; ++r) {
         if (q_len[r] <= 1) continue;
@@ -182,8 +211,10 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
     pl->prefill_cta_start.clear();
     if (tiles.empty()) return;
 
-    // cut[i] = key-tile indices at which tile i is cut into pieces (ascending, exclusive of 0 and key_tiles)
-    std::vector<std::vector<int>> cuts(tiles.size());
+    // (tile, key-tile index) of every cut, ascending in both: tile i is cut into pieces at these key tiles
+    // (exclusive of 0 and key_tiles)
+    struct Cut { int tile, at; };
+    std::vector<Cut> cuts;
     // owner CTA of the first piece of each tile and of each following piece, for the static partition
     bool static_partition = false, whole_items = false;
     if (opts && opts->prefill_segment_tokens > 0) {
@@ -195,7 +226,7 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
             int kt0 = 0;
             for (int s = 0; s + 1 < n_seg; ++s) {
                 kt0 += base_tiles + (s < extra ? 1 : 0);
-                cuts[i].push_back(kt0);
+                cuts.push_back(Cut{(int)i, kt0});
             }
         }
     } else if ((int64_t)tiles.size() < 4LL * pl->pf_sms) {
@@ -212,27 +243,28 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
             std::vector<int> order(tiles.size());
             for (size_t i = 0; i < tiles.size(); ++i) order[i] = (int)i;
             std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return tiles[a].key_tiles > tiles[b].key_tiles; });
-            std::vector<double> load(n_cta, 0.0);
+            // (least work so far, CTA): equal loads go to the lower CTA
+            typedef std::pair<double, int> Slot;
+            std::vector<Slot> heap((size_t)n_cta);
+            for (int c = 0; c < n_cta; ++c) heap[c] = Slot(0.0, c);  // ascending: already a min-heap under greater<>
             std::vector<int> owner(tiles.size());
-            // a heap would do; CTAs are at most 148 and items a few hundred
+            std::vector<int32_t> count((size_t)n_cta + 1, 0);
+            double makespan = 0;
             for (int i : order) {
-                int best = 0;
-                for (int c = 1; c < n_cta; ++c)
-                    if (load[c] < load[best]) best = c;
-                owner[i] = best;
-                load[best] += kPrefillFixedCost + tiles[i].key_tiles + kPrefillMaskedExtra;
+                std::pop_heap(heap.begin(), heap.end(), std::greater<Slot>());
+                Slot& least = heap.back();
+                owner[i] = least.second;
+                ++count[least.second + 1];
+                least.first += kPrefillFixedCost + tiles[i].key_tiles + kPrefillMaskedExtra;
+                makespan = std::max(makespan, least.first);
+                std::push_heap(heap.begin(), heap.end(), std::greater<Slot>());
             }
-            const double makespan = *std::max_element(load.begin(), load.end());
             // (cutting is not free either: the merge kernel and the partial rows cost about kPrefillCutCost steps)
             if (makespan <= std::max(kPrefillWholeItemSlack * total / n_cta, total / n_cta + kPrefillCutCost)) {
-                std::vector<Tile> sorted;
-                sorted.reserve(tiles.size());
-                pl->prefill_cta_start.assign(1, 0);
-                for (int c = 0; c < n_cta; ++c) {
-                    for (int i : order)
-                        if (owner[i] == c) sorted.push_back(tiles[i]);
-                    pl->prefill_cta_start.push_back((int32_t)sorted.size());
-                }
+                for (int c = 0; c < n_cta; ++c) count[c + 1] += count[c];
+                pl->prefill_cta_start.assign(count.begin(), count.end());
+                std::vector<Tile> sorted(tiles.size());
+                for (int i : order) sorted[(size_t)count[owner[i]]++] = tiles[i];  // each CTA's items longest first
                 tiles.swap(sorted);
                 whole_items = true;
             }
@@ -247,7 +279,7 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
         for (int pass = 0; pass < 7; ++pass) {
             const double quota = pass == 6 ? q_hi : 0.5 * (q_lo + q_hi);  // the last pass keeps a quota known to fit
             pl->prefill_cta_start.assign(1, 0);
-            for (auto& c : cuts) c.clear();
+            cuts.clear();
             n_items = 0;
             int cta = 0;
             double cum = 0, cum_at_last = 0;  // cost handed out so far; and before the last CTA
@@ -263,7 +295,8 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
                     const double rest = kPrefillFixedCost + (kt - kt0) + kPrefillMaskedExtra;  // the item's remaining tiles as one piece
                     const double room = (cta + 1) * quota - cum;
                     const bool cta_has_work = pl->prefill_cta_start.back() < n_items;
-                    const int take = (int)std::lround(room - kPrefillFixedCost);
+                    const double fit = room - kPrefillFixedCost;
+                    const int take = fit < 0.5 ? 0 : (int)(fit + 0.5);  // key tiles that fit, to the nearest
                     if (cta == n_cta - 1 || rest <= room + 0.5 || take >= kt - kt0 || (take < 1 && !cta_has_work)) {
                         cum += rest;
                         ++n_items;
@@ -271,7 +304,7 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
                     }
                     if (take >= 1) {
                         kt0 += take;
-                        cuts[i].push_back(kt0);
+                        cuts.push_back(Cut{(int)i, kt0});
                         cum += kPrefillFixedCost + take;
                         ++n_items;
                     }
@@ -287,9 +320,13 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
         }
     }
 
+    pl->prefill.reserve(tiles.size() + cuts.size());
+    size_t next_cut = 0;
     for (size_t i = 0; i < tiles.size(); ++i) {
         const Tile& t = tiles[i];
-        const int n_seg = (int)cuts[i].size() + 1;
+        const size_t first_cut = next_cut;
+        while (next_cut < cuts.size() && cuts[next_cut].tile == (int)i) ++next_cut;
+        const int n_seg = (int)(next_cut - first_cut) + 1;
         const int visible = t.first_pos + t.n_tok;
         int32_t slot_base = -1;
         if (n_seg > 1) {
@@ -305,8 +342,8 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
             *n_slots += (int64_t)n_seg * t.n_tok * G;
         }
         for (int s = 0; s < n_seg; ++s) {
-            const int kt0 = s == 0 ? 0 : cuts[i][s - 1];
-            const int kt1 = s == n_seg - 1 ? t.key_tiles : cuts[i][s];
+            const int kt0 = s == 0 ? 0 : cuts[first_cut + s - 1].at;
+            const int kt1 = s == n_seg - 1 ? t.key_tiles : cuts[first_cut + s].at;
             PrefillItem it{};
             it.req = t.r;
             it.kv_head = t.g;
@@ -378,11 +415,8 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
         if (fresh) delete pl;
         return fail(PS_ERR_CUDA, "no CUDA device to plan for (pass opts->num_sms to plan without one)");
     }
-    pl->pieces.clear();
-    pl->units.clear();
     pl->prefill.clear();
     pl->merge.clear();
-    pl->dmerge.clear();
     pl->decode_merge_rows = 0;
     pl->prior.assign(prior_host, prior_host + n);
     pl->info = ps_plan_info{};
