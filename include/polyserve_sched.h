@@ -70,6 +70,42 @@ typedef struct ps_table ps_table; /* (token batch, KV tokens, prefill work) -> m
 ps_status ps_table_build(const ps_grid_row *rows, int64_t n_rows, ps_table **out);
 
 /*
+ * The same sweep fitted in the overlap form.  This library runs the decode
+ * rows and the prefill chunk of a mixed batch side by side on disjoint SMs, so
+ * a mixed batch takes about as long as the slower of its two parts, not their
+ * sum (section 3.4 adds the terms for engines that run them one after the
+ * other).  A line of an overlap table predicts
+ *     latency_us = base + max(decode_intercept + slope_kv * kv_tokens,
+ *                             prefill_intercept + slope_pf * prefill_flops),
+ * with the prefill term left out when prefill_flops = 0 and the decode term
+ * when kv_tokens = 0; base is 0 after this call and takes what
+ * ps_table_add_batch_term adds.  The four parameters are fitted once over all
+ * rows (every line of the table, one per distinct token_batch, carries the
+ * same four) by alternating least squares:
+ *   1. the sum form a + s kv + q pf over all rows (rules of ps_table_build)
+ *      gives the start: decode_intercept = prefill_intercept = a, s, q (a
+ *      negative slope is taken as 0);
+ *   2. a row belongs to the decode side if its prefill_flops = 0, to the
+ *      prefill side if its kv_tokens = 0, else to the side whose term (at the
+ *      start: s kv against q pf; later the whole term with its intercept) is
+ *      the larger, ties to the decode side;
+ *   3. decode side first, then prefill side: least-squares line of latency
+ *      over that side's own regressor on that side's rows; a side with fewer
+ *      than two rows, or whose regressor does not vary, keeps its parameters;
+ *   4. rows are assigned again (step 2); repeat 3-4 until no row moves, at
+ *      most 64 times.
+ * ps_table_get_lines returns base and the two slopes of such a table,
+ * ps_table_get_overlap whether a table is in this form and the two intercepts
+ * (outputs may be NULL; capacity in lines; for a sum-form table only
+ * *is_overlap_out = 0 is written).  ps_table_scale multiplies all five
+ * coefficients; prediction, admission and chunk prediction use whichever form
+ * the table has.  Errors as for ps_table_build.
+ */
+ps_status ps_table_build_overlap(const ps_grid_row *rows, int64_t n_rows, ps_table **out);
+ps_status ps_table_get_overlap(const ps_table *table, int32_t *is_overlap_out, double *decode_intercept_us_out,
+                               double *prefill_intercept_us_out, int32_t capacity);
+
+/*
  * Build a table from explicit lines: line i predicts intercept_us[i] +
  * slope_us_per_token[i] * kv_tokens + slope_us_per_flop[i] * prefill_flops at
  * batch size token_batch[i] (slope_us_per_flop == NULL: all zero).  The lines

@@ -61,7 +61,18 @@ def table_predict(lines, token_batch, kv_tokens, prefill_flops=0.0):
     """Predicted iteration time: the line of that batch size evaluated at (kv_tokens, prefill_flops); between two
     lines their two values interpolated linearly in the batch size; outside the lines the nearest line as it is."""
     lines = sorted(lines)
-    at = lambda ln: ln[1] + ln[2] * float(kv_tokens) + ln[3] * float(prefill_flops)
+
+    def at(ln):
+        if len(ln) == 4:  # sum form
+            return ln[1] + ln[2] * float(kv_tokens) + ln[3] * float(prefill_flops)
+        _, base, a_d, s, a_p, q = ln  # overlap form, see table_build_overlap
+        dec, pre = a_d + s * float(kv_tokens), a_p + q * float(prefill_flops)
+        if prefill_flops == 0:
+            return base + dec
+        if kv_tokens == 0:
+            return base + pre
+        return base + max(dec, pre)
+
     if token_batch <= lines[0][0]:
         return at(lines[0])
     if token_batch >= lines[-1][0]:
@@ -71,6 +82,55 @@ def table_predict(lines, token_batch, kv_tokens, prefill_flops=0.0):
             w = (token_batch - lo[0]) / float(hi[0] - lo[0])
             return at(lo) + (at(hi) - at(lo)) * w
     raise AssertionError("unreachable")
+
+
+def table_build_overlap(rows):
+    """The sweep fitted for an engine that runs the decode rows and the prefill chunk of a batch side by side: a
+    mixed batch then takes about as long as the slower part, latency = base + max(a_d + s kv_tokens, a_p + q
+    prefill_flops), the prefill term absent without a chunk and the decode term without KV tokens (section 3.4 adds
+    the terms, for parts that run one after the other).  One set of four parameters for the whole sweep, found by
+    alternating least squares: start from the sum form fitted over all rows (a_d = a_p = its intercept, a negative
+    slope taken as 0); give each
+    row to the side whose term is larger (rows without prefill work to the decode side, rows without KV tokens to
+    the prefill side, ties to the decode side; at the start the terms are compared without intercepts); fit each
+    side's line on its own rows and its own regressor (a side with fewer than two rows or a constant regressor
+    keeps what it has), decode side first; assign again; stop when no row moves or after 64 rounds.  Returns one
+    line (token_batch, base = 0, a_d, s, a_p, q) per distinct batch size, all with the same four parameters."""
+    rows = [(int(b), float(kv), float(pf), float(lat)) for b, kv, pf, lat in rows]
+    (_, a, s, q), = table_build([(1, kv, pf, lat) for _, kv, pf, lat in rows])
+    a_d = a_p = a
+    s, q = max(s, 0.0), max(q, 0.0)
+
+    def side(kv, pf, dec, pre):
+        if pf == 0.0:
+            return "decode"
+        if kv == 0.0:
+            return "prefill"
+        return "decode" if dec >= pre else "prefill"
+
+    sides = [side(kv, pf, s * kv, q * pf) for _, kv, pf, _ in rows]
+    for _ in range(64):
+        for which in ("decode", "prefill"):
+            pts = [((kv if which == "decode" else pf), lat) for (_, kv, pf, lat), z in zip(rows, sides) if z == which]
+            if len(pts) < 2:
+                continue
+            mx = sum(x for x, _ in pts) / len(pts)
+            my = sum(y for _, y in pts) / len(pts)
+            sxx = sum((x - mx) * (x - mx) for x, _ in pts)
+            sxy = sum((x - mx) * (y - my) for x, y in pts)
+            if not sxx > 0.0:
+                continue
+            if which == "decode":
+                s = sxy / sxx
+                a_d = my - s * mx
+            else:
+                q = sxy / sxx
+                a_p = my - q * mx
+        again = [side(kv, pf, a_d + s * kv, a_p + q * pf) for _, kv, pf, _ in rows]
+        if again == sides:
+            break
+        sides = again
+    return [(b, 0.0, a_d, s, a_p, q) for b in sorted({b for b, _, _, _ in rows})]
 
 
 def table_add_batch_term(lines, samples):
@@ -89,12 +149,12 @@ def table_add_batch_term(lines, samples):
                 return lo[1] + (hi[1] - lo[1]) * ((b - lo[0]) / float(hi[0] - lo[0]))
         raise AssertionError("unreachable")
 
-    return [(b, a + term(b), s, q) for b, a, s, q in lines]
+    return [(ln[0], ln[1] + term(ln[0])) + tuple(ln[2:]) for ln in lines]
 
 
 def table_scale(lines, factor):
     """Every coefficient times factor (a model of n identical layers is n times one layer)."""
-    return [(b, a * factor, s * factor, q * factor) for b, a, s, q in lines]
+    return [(ln[0],) + tuple(c * factor for c in ln[1:]) for ln in lines]
 
 
 # ---------------------------------------------------------------------------

@@ -12,7 +12,8 @@ from .binding import (  # noqa: F401
     ps_plan_get_timing, ps_plan_opts, ps_plan_set_timing, ps_plan_status, ps_profile_grid, ps_shape, ps_version,
 )
 from .sched_binding import (  # noqa: F401
-    ps_admit, ps_chunk_next, ps_chunk_predict, ps_chunk_schedule, ps_peak_kv, ps_table_add_batch_term, ps_table_build, ps_table_free,
+    ps_admit, ps_chunk_next, ps_chunk_predict, ps_chunk_schedule, ps_peak_kv, ps_table_add_batch_term, ps_table_build, ps_table_build_overlap, ps_table_free,
+    ps_table_get_overlap,
     ps_table_from_lines, ps_table_scale,
     ps_table_get_lines, ps_table_predict, ps_table_size,
 )

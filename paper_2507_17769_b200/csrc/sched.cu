@@ -15,13 +15,61 @@ struct ps_table {
     std::vector<double> intercept;
     std::vector<double> slope;     // microseconds per KV token
     std::vector<double> slope_pf;  // microseconds per flop of prefill attention
+    // Overlap form (decode and prefill attention side by side): a line is intercept + max(dec_icpt + slope kv,
+    // pf_icpt + slope_pf pf); `intercept` then holds only what depends on the batch size alone.
+    bool overlap = false;
+    std::vector<double> dec_icpt, pf_icpt;
 };
 
 namespace ps {
 namespace {
 
 double line_at(const ps_table& t, size_t i, int64_t kv, double pf) {
-    return t.intercept[i] + t.slope[i] * (double)kv + t.slope_pf[i] * pf;
+    if (!t.overlap) return t.intercept[i] + t.slope[i] * (double)kv + t.slope_pf[i] * pf;
+    const double dec = t.dec_icpt[i] + t.slope[i] * (double)kv, pre = t.pf_icpt[i] + t.slope_pf[i] * pf;
+    // a batch without a chunk runs no prefill kernel, one without KV tokens no decode kernel
+    const double attn = pf == 0.0 ? dec : kv == 0 ? pre : std::max(dec, pre);
+    return t.intercept[i] + attn;
+}
+
+// Least squares of y = a + s x + q p over the rows listed in idx (centred sums; a regressor that does not vary, or
+// the second of two collinear ones, is left out).
+struct Plane { double a, s, q; };
+Plane fit_plane(const ps_grid_row* rows, const int64_t* idx, int64_t n_idx) {
+    const double n = (double)n_idx;
+    double sum_x = 0.0, sum_p = 0.0, sum_y = 0.0;
+    for (int64_t k = 0; k < n_idx; ++k) {
+        const ps_grid_row& r = rows[idx[k]];
+        sum_x += (double)r.kv_tokens, sum_p += r.prefill_flops, sum_y += (double)r.latency_us;
+    }
+    const double mx = sum_x / n, mp = sum_p / n, my = sum_y / n;
+    double sxx = 0.0, spp = 0.0, sxp = 0.0, sxy = 0.0, spy = 0.0;
+    for (int64_t k = 0; k < n_idx; ++k) {
+        const ps_grid_row& r = rows[idx[k]];
+        const double dx = (double)r.kv_tokens - mx, dp = r.prefill_flops - mp, dy = (double)r.latency_us - my;
+        sxx += dx * dx, spp += dp * dp, sxp += dx * dp, sxy += dx * dy, spy += dp * dy;
+    }
+    const double det = sxx * spp - sxp * sxp;
+    Plane f{0.0, 0.0, 0.0};
+    if (sxx > 0.0 && spp > 0.0 && det > 1e-9 * sxx * spp) {
+        f.s = (sxy * spp - spy * sxp) / det;
+        f.q = (spy * sxx - sxy * sxp) / det;
+    } else if (sxx > 0.0) {
+        f.s = sxy / sxx;
+    } else if (spp > 0.0) {
+        f.q = spy / spp;
+    }
+    f.a = my - f.s * mx - f.q * mp;
+    return f;
+}
+
+ps_status check_rows(const char* who, const ps_grid_row* rows, int64_t n_rows) {
+    for (int64_t i = 0; i < n_rows; ++i)
+        if (rows[i].token_batch < 1 || rows[i].kv_tokens < 0 || !std::isfinite(rows[i].latency_us) || !std::isfinite(rows[i].prefill_flops) ||
+            rows[i].prefill_flops < 0.0)
+            return fail(PS_ERR_INVALID, "%s: row %lld has token_batch %d, kv_tokens %lld, latency %g", who, (long long)i,
+                        rows[i].token_batch, (long long)rows[i].kv_tokens, (double)rows[i].latency_us);
+    return PS_OK;
 }
 
 double predict(const ps_table& t, int32_t token_batch, int64_t kv, double pf) {
@@ -120,11 +168,7 @@ ps_status ps_table_from_lines(const int32_t* token_batch, const double* intercep
 ps_status ps_table_build(const ps_grid_row* rows, int64_t n_rows, ps_table** out) {
     ps::clear_error();
     if (!rows || !out || n_rows < 1) return fail(PS_ERR_INVALID, "ps_table_build: null pointer or n_rows < 1");
-    for (int64_t i = 0; i < n_rows; ++i)
-        if (rows[i].token_batch < 1 || rows[i].kv_tokens < 0 || !std::isfinite(rows[i].latency_us) || !std::isfinite(rows[i].prefill_flops) ||
-            rows[i].prefill_flops < 0.0)
-            return fail(PS_ERR_INVALID, "ps_table_build: row %lld has token_batch %d, kv_tokens %lld, latency %g", (long long)i,
-                        rows[i].token_batch, (long long)rows[i].kv_tokens, (double)rows[i].latency_us);
+    if (ps_status st = ps::check_rows("ps_table_build", rows, n_rows)) return st;
     // rows of one batch size together, in their input order
     std::vector<int64_t> order(n_rows);
     std::iota(order.begin(), order.end(), (int64_t)0);
@@ -134,38 +178,93 @@ ps_status ps_table_build(const ps_grid_row* rows, int64_t n_rows, ps_table** out
     for (int64_t g0 = 0; g0 < n_rows;) {
         int64_t g1 = g0;
         while (g1 < n_rows && rows[order[g1]].token_batch == rows[order[g0]].token_batch) ++g1;
-        const double n = (double)(g1 - g0);
-        double sum_x = 0.0, sum_p = 0.0, sum_y = 0.0;
-        for (int64_t k = g0; k < g1; ++k) {
-            const ps_grid_row& r = rows[order[k]];
-            sum_x += (double)r.kv_tokens, sum_p += r.prefill_flops, sum_y += (double)r.latency_us;
-        }
-        const double mx = sum_x / n, mp = sum_p / n, my = sum_y / n;
-        double sxx = 0.0, spp = 0.0, sxp = 0.0, sxy = 0.0, spy = 0.0;
-        for (int64_t k = g0; k < g1; ++k) {
-            const ps_grid_row& r = rows[order[k]];
-            const double dx = (double)r.kv_tokens - mx, dp = r.prefill_flops - mp, dy = (double)r.latency_us - my;
-            sxx += dx * dx, spp += dp * dp, sxp += dx * dp, sxy += dx * dy, spy += dp * dy;
-        }
-        // normal equations of latency = a + s kv + q pf on centred sums; a regressor that does not vary within the
-        // line, or the second of two collinear ones, is left out
-        const double det = sxx * spp - sxp * sxp;
-        double s_kv = 0.0, s_pf = 0.0;
-        if (sxx > 0.0 && spp > 0.0 && det > 1e-9 * sxx * spp) {
-            s_kv = (sxy * spp - spy * sxp) / det;
-            s_pf = (spy * sxx - sxy * sxp) / det;
-        } else if (sxx > 0.0) {
-            s_kv = sxy / sxx;
-        } else if (spp > 0.0) {
-            s_pf = spy / spp;
-        }
+        const ps::Plane f = ps::fit_plane(rows, order.data() + g0, g1 - g0);
         batch.push_back(rows[order[g0]].token_batch);
-        slope.push_back(s_kv);
-        slope_pf.push_back(s_pf);
-        icpt.push_back(my - s_kv * mx - s_pf * mp);
+        slope.push_back(f.s);
+        slope_pf.push_back(f.q);
+        icpt.push_back(f.a);
         g0 = g1;
     }
     return ps_table_from_lines(batch.data(), icpt.data(), slope.data(), slope_pf.data(), (int32_t)batch.size(), out);
+}
+
+ps_status ps_table_build_overlap(const ps_grid_row* rows, int64_t n_rows, ps_table** out) {
+    ps::clear_error();
+    if (!rows || !out || n_rows < 1) return fail(PS_ERR_INVALID, "ps_table_build_overlap: null pointer or n_rows < 1");
+    if (ps_status st = ps::check_rows("ps_table_build_overlap", rows, n_rows)) return st;
+    std::vector<int64_t> all(n_rows);
+    std::iota(all.begin(), all.end(), (int64_t)0);
+    // start from the sum form over all rows: each row goes to the side whose term is the larger one there
+    const ps::Plane sum = ps::fit_plane(rows, all.data(), n_rows);
+    // (a slope below zero at the start would let that term fall with the work; it is taken as zero until fitted)
+    double a_d = sum.a, s = std::max(sum.s, 0.0), a_p = sum.a, q = std::max(sum.q, 0.0);
+    std::vector<char> on_decode(n_rows);
+    auto side = [&](int64_t i, double dec, double pre) -> char {
+        if (rows[i].prefill_flops == 0.0) return 1;
+        if (rows[i].kv_tokens == 0) return 0;
+        return dec >= pre ? 1 : 0;
+    };
+    for (int64_t i = 0; i < n_rows; ++i) on_decode[i] = side(i, s * (double)rows[i].kv_tokens, q * rows[i].prefill_flops);
+    std::vector<int64_t> idx;
+    for (int pass = 0; pass < 64; ++pass) {
+        // one regressor per side: the other one's column is hidden from the fit
+        for (int which = 1; which >= 0; --which) {
+            idx.clear();
+            for (int64_t i = 0; i < n_rows; ++i)
+                if (on_decode[i] == which) idx.push_back(i);
+            if (idx.size() < 2) continue;  // keeps the parameters it has
+            const double n = (double)idx.size();
+            double sum_x = 0.0, sum_y = 0.0;
+            for (int64_t i : idx) sum_x += which ? (double)rows[i].kv_tokens : rows[i].prefill_flops, sum_y += (double)rows[i].latency_us;
+            const double mx = sum_x / n, my = sum_y / n;
+            double sxx = 0.0, sxy = 0.0;
+            for (int64_t i : idx) {
+                const double dx = (which ? (double)rows[i].kv_tokens : rows[i].prefill_flops) - mx;
+                sxx += dx * dx, sxy += dx * ((double)rows[i].latency_us - my);
+            }
+            if (!(sxx > 0.0)) continue;
+            const double slope = sxy / sxx;
+            if (which) s = slope, a_d = my - slope * mx;
+            else q = slope, a_p = my - slope * mx;
+        }
+        bool changed = false;
+        for (int64_t i = 0; i < n_rows; ++i) {
+            const char now = side(i, a_d + s * (double)rows[i].kv_tokens, a_p + q * rows[i].prefill_flops);
+            changed = changed || now != on_decode[i];
+            on_decode[i] = now;
+        }
+        if (!changed) break;
+    }
+    std::vector<int32_t> batch(n_rows);
+    for (int64_t i = 0; i < n_rows; ++i) batch[i] = rows[i].token_batch;
+    std::sort(batch.begin(), batch.end());
+    batch.erase(std::unique(batch.begin(), batch.end()), batch.end());
+    ps_table* t = new (std::nothrow) ps_table;
+    if (!t) return fail(PS_ERR_OOM, "ps_table_build_overlap: out of host memory");
+    const size_t n_lines = batch.size();
+    t->batch = batch;
+    t->overlap = true;
+    t->intercept.assign(n_lines, 0.0);
+    t->dec_icpt.assign(n_lines, a_d);
+    t->slope.assign(n_lines, s);
+    t->pf_icpt.assign(n_lines, a_p);
+    t->slope_pf.assign(n_lines, q);
+    *out = t;
+    return PS_OK;
+}
+
+ps_status ps_table_get_overlap(const ps_table* table, int32_t* is_overlap_out, double* decode_intercept_us_out,
+                               double* prefill_intercept_us_out, int32_t capacity) {
+    ps::clear_error();
+    if (!table || !is_overlap_out) return fail(PS_ERR_INVALID, "ps_table_get_overlap: null pointer");
+    *is_overlap_out = table->overlap ? 1 : 0;
+    if (!table->overlap || (!decode_intercept_us_out && !prefill_intercept_us_out)) return PS_OK;
+    if (capacity < (int32_t)table->batch.size()) return fail(PS_ERR_INVALID, "ps_table_get_overlap: capacity %d < %zu lines", capacity, table->batch.size());
+    for (size_t i = 0; i < table->batch.size(); ++i) {
+        if (decode_intercept_us_out) decode_intercept_us_out[i] = table->dec_icpt[i];
+        if (prefill_intercept_us_out) prefill_intercept_us_out[i] = table->pf_icpt[i];
+    }
+    return PS_OK;
 }
 
 ps_status ps_table_free(ps_table* table) {
@@ -209,6 +308,7 @@ ps_status ps_table_scale(ps_table* table, double factor) {
         table->intercept[l] *= factor;
         table->slope[l] *= factor;
         table->slope_pf[l] *= factor;
+        if (table->overlap) table->dec_icpt[l] *= factor, table->pf_icpt[l] *= factor;
     }
     return PS_OK;
 }

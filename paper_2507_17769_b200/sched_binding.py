@@ -11,7 +11,7 @@ import numpy as np
 
 from . import binding as B
 
-EXPORTS = ["ps_table_build", "ps_table_from_lines", "ps_table_free", "ps_table_add_batch_term", "ps_table_scale", "ps_table_size",
+EXPORTS = ["ps_table_build", "ps_table_build_overlap", "ps_table_get_overlap", "ps_table_from_lines", "ps_table_free", "ps_table_add_batch_term", "ps_table_scale", "ps_table_size",
            "ps_table_get_lines",
            "ps_table_predict", "ps_peak_kv", "ps_admit", "ps_chunk_next", "ps_chunk_schedule", "ps_chunk_predict"]
 
@@ -25,6 +25,8 @@ def _lib():
     lib = B.load()
     if not _ready:
         lib.ps_table_build.argtypes = [ctypes.POINTER(B.ps_grid_row), _i64, ctypes.POINTER(_vp)]
+        lib.ps_table_build_overlap.argtypes = [ctypes.POINTER(B.ps_grid_row), _i64, ctypes.POINTER(_vp)]
+        lib.ps_table_get_overlap.argtypes = [_vp, ctypes.POINTER(_i32), _f64p, _f64p, _i32]
         lib.ps_table_from_lines.argtypes = [_i32p, _f64p, _f64p, _f64p, _i32, ctypes.POINTER(_vp)]
         lib.ps_table_free.argtypes = [_vp]
         lib.ps_table_add_batch_term.argtypes = [_vp, _i32p, _f64p, _i32]
@@ -56,6 +58,26 @@ def ps_table_build(rows):
     out = _vp(0)
     B._check(_lib().ps_table_build(arr, len(rows), ctypes.byref(out)))
     return out.value
+
+
+def ps_table_build_overlap(rows):
+    """The sweep fitted as base + max(decode term, prefill term) (one set of parameters for all lines)."""
+    arr = (B.ps_grid_row * len(rows))(*rows)
+    out = _vp(0)
+    B._check(_lib().ps_table_build_overlap(arr, len(rows), ctypes.byref(out)))
+    return out.value
+
+
+def ps_table_get_overlap(table):
+    """Returns None for a sum-form table, else (decode_intercept_us, prefill_intercept_us: float64[n])."""
+    flag = _i32(0)
+    B._check(_lib().ps_table_get_overlap(table, ctypes.byref(flag), None, None, 0))
+    if not flag.value:
+        return None
+    n = ps_table_size(table)
+    a_d, a_p = np.zeros(n, np.float64), np.zeros(n, np.float64)
+    B._check(_lib().ps_table_get_overlap(table, ctypes.byref(flag), a_d.ctypes.data_as(_f64p), a_p.ctypes.data_as(_f64p), n))
+    return a_d, a_p
 
 
 def ps_table_from_lines(token_batch, intercept_us, slope_us_per_token, slope_us_per_flop=None):

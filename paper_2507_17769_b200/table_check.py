@@ -6,7 +6,9 @@
    least-squares fit of latency over KV tokens and prefill-attention work).
 2. A second sweep over batch shapes that are not on the grid, with other seeds; each of its draws is timed and
    compared with ps_table_predict(token_batch, kv_tokens, prefill_flops), and with the same table looked up by the
-   paper's two keys alone (prefill work left out of the fit).  Prints the relative prediction errors.
+   paper's two keys alone (prefill work left out of the fit), and with the overlap form ps_table_build_overlap fits
+   to the same sweep (base + max(decode term, prefill term): the two kernels of a mixed batch run side by side).
+   Prints the relative prediction errors.
 3. The host cost of the admission test (ps_admit) and of the chunk prediction (ps_chunk_predict) for an instance
    with 256 running requests, in decisions per second through this binding.
 4. With --iteration: the whole-iteration table of the paper's model T_iter = GEMM(B) + decode attention + prefill
@@ -151,12 +153,19 @@ def main():
                     "chunk_768_up": summary(err[heavy]) if heavy.any() else None}
 
         blind = two_key_table(rows)
+        overlap = S.ps_table_build_overlap(rows)
         try:
+            _, _, o_s, o_q = S.ps_table_get_lines(overlap)
+            o_ad, o_ap = S.ps_table_get_overlap(overlap)
+            print("overlap form: latency_us = max(%.2f + %.4e * kv_tokens, %.2f + %.4e * prefill_flops)" % (o_ad[0], o_s[0], o_ap[0], o_q[0]))
             report = {"fit_rows": summary(rel_errors(table, rows)), "held_out": split(rel_errors(table, test)),
                       "fit_rows_two_keys": summary(rel_errors(blind, rows, False)),
-                      "held_out_two_keys": split(rel_errors(blind, test, False)), "host": host_rates(table)}
+                      "held_out_two_keys": split(rel_errors(blind, test, False)),
+                      "fit_rows_overlap": summary(rel_errors(overlap, rows)), "held_out_overlap": split(rel_errors(overlap, test)),
+                      "host": host_rates(table), "host_overlap": host_rates(overlap)}
         finally:
             S.ps_table_free(blind)
+            S.ps_table_free(overlap)
         print(json.dumps(report))
         if a.iteration:
             S.ps_table_free(iteration_table(shape, grid, seeds, a.warmup, a.iters))

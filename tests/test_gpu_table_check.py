@@ -25,5 +25,13 @@ def test_table_from_a_sweep_predicts_held_out_decode_heavy_batches():
         ok, pred, peak = S.ps_admit(table, kv, rem, 2048, 100, 0, 0, 0.0, 1e9)
         assert ok and peak == 64 * (2048 + 99)
         assert not S.ps_admit(table, kv, rem, 2048, 100, 0, 0, 0.0, pred * 0.99)[0]
+        # the same sweep in the overlap form: positive slopes on both sides, held-out batches within the same bound
+        overlap = S.ps_table_build_overlap(rows)
+        try:
+            _, base, o_s, o_q = S.ps_table_get_lines(overlap)
+            assert (base == 0).all() and (o_s > 0).all() and (o_q >= 0).all() and S.ps_table_get_overlap(overlap) is not None
+            assert np.median(np.abs(rel_errors(overlap, held))) < 0.5
+        finally:
+            S.ps_table_free(overlap)
     finally:
         S.ps_table_free(table)

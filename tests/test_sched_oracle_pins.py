@@ -242,3 +242,71 @@ def test_chunk_prediction_closed_form():
     want = sum(g * phi * (min(c, 5000 - k * c) * k * c + 0.5 * min(c, 5000 - k * c) * (min(c, 5000 - k * c) + 1)) for k in range(iters))
     assert total == pytest.approx(want)
     assert so.prefill_work(4.0 * 128 * 32, 1536, 3885) == 4 * 128 * 32 * (1536 * 3885 + 1536 * 1537 // 2)
+
+
+# ---------------------------------------------------------------------------
+# overlap form: base + max(decode term, prefill term)
+# ---------------------------------------------------------------------------
+def overlap_rows(rng, a_d, s, a_p, q, n=400, noise=0.0):
+    rows = []
+    for i in range(n):
+        kv = float(rng.integers(2_000, 2_000_000))
+        pf = float(rng.uniform(1e9, 1.2e12))
+        if i % 10 == 0:
+            pf = 0.0  # decode-only batches
+        if i % 10 == 1:
+            kv = 0.0  # a chunk alone
+        dec, pre = a_d + s * kv, a_p + q * pf
+        lat = dec if pf == 0.0 else pre if kv == 0.0 else max(dec, pre)
+        rows.append((int(rng.choice([72, 320, 1032])), kv, pf, lat * (1.0 + noise * rng.standard_normal())))
+    return rows
+
+
+def test_overlap_fit_recovers_an_exact_max_of_two_lines():
+    rng = np.random.default_rng(11)
+    a_d, s, a_p, q = 26.0, 6.1e-4, 34.0, 9.9e-10
+    lines = so.table_build_overlap(overlap_rows(rng, a_d, s, a_p, q))
+    assert [ln[0] for ln in lines] == [72, 320, 1032]
+    for ln in lines:
+        assert ln[1] == 0.0
+        np.testing.assert_allclose(ln[2:], (a_d, s, a_p, q), rtol=1e-9)
+    # with 3 % noise on the latencies the parameters come back within a few per cent, the slopes within one
+    noisy = so.table_build_overlap(overlap_rows(np.random.default_rng(12), a_d, s, a_p, q, n=3000, noise=0.03))[0]
+    np.testing.assert_allclose(noisy[3], s, rtol=0.02)
+    np.testing.assert_allclose(noisy[5], q, rtol=0.02)
+
+
+def test_overlap_fit_without_chunks_is_the_plain_regression_line():
+    """No row carries prefill work: every row is on the decode side and the fit is numpy's straight line."""
+    rng = np.random.default_rng(13)
+    kv = rng.integers(1_000, 3_000_000, 60).astype(np.float64)
+    lat = 20.0 + 6e-4 * kv + rng.normal(0.0, 3.0, 60)
+    (ln,) = so.table_build_overlap([(256, x, 0.0, y) for x, y in zip(kv, lat)])
+    slope, icpt = np.polyfit(kv, lat, 1)
+    np.testing.assert_allclose((ln[2], ln[3]), (icpt, slope), rtol=1e-8)
+    # and the other way round: chunks alone
+    pf = rng.uniform(1e9, 1e12, 60)
+    lat = 30.0 + 1e-9 * pf + rng.normal(0.0, 3.0, 60)
+    (ln,) = so.table_build_overlap([(256, 0.0, x, y) for x, y in zip(pf, lat)])
+    slope, icpt = np.polyfit(pf, lat, 1)
+    np.testing.assert_allclose((ln[4], ln[5]), (icpt, slope), rtol=1e-8)
+
+
+def test_overlap_lookup_by_hand():
+    lines = [(64, 5.0, 10.0, 1e-3, 20.0, 1e-9), (128, 9.0, 10.0, 1e-3, 20.0, 1e-9)]
+    # decode side larger: 5 + max(10 + 100, 20 + 50); prefill side larger; a batch without a chunk; a chunk alone
+    assert so.table_predict(lines, 64, 100_000, 5e10) == pytest.approx(115.0, rel=1e-12)
+    assert so.table_predict(lines, 64, 10_000, 5e10) == pytest.approx(75.0, rel=1e-12)
+    assert so.table_predict(lines, 64, 1_000, 0.0) == pytest.approx(16.0, rel=1e-12)  # not max(11, 20)
+    assert so.table_predict(lines, 64, 0, 1e9) == pytest.approx(26.0, rel=1e-12)  # not max(10, 21)
+    assert so.table_predict(lines, 96, 100_000, 5e10) == pytest.approx(117.0, rel=1e-12)  # half way between the bases
+    # never above the sum of the two terms, never below either; the batch term and the scaling act on it as on a sum table
+    rng = np.random.default_rng(14)
+    for _ in range(200):
+        kv, pf = int(rng.integers(1, 10**6)), float(rng.uniform(1.0, 1e12))
+        t = so.table_predict(lines, 64, kv, pf)
+        dec, pre = 10.0 + 1e-3 * kv, 20.0 + 1e-9 * pf
+        assert max(dec, pre) + 5.0 == pytest.approx(t, rel=1e-12) and t <= 5.0 + dec + pre
+    more = so.table_scale(so.table_add_batch_term(lines, [(64, 100.0), (128, 300.0)]), 32.0)
+    assert so.table_predict(more, 64, 100_000, 5e10) == pytest.approx(32.0 * 215.0, rel=1e-12)
+    assert so.table_predict(more, 128, 100_000, 5e10) == pytest.approx(32.0 * 419.0, rel=1e-12)

@@ -108,6 +108,85 @@ def test_batch_term_and_scale_match_the_oracle():
             S.ps_table_free(t)
 
 
+def overlap_grid_rows(rng, n, with_pure=True):
+    """Sweep-like rows of an engine that overlaps the two parts: latency ~ max(decode term, prefill term), 4 % noise."""
+    rows, plain = [], []
+    for i in range(n):
+        b = int(rng.choice([72, 96, 320, 1032, 2304]))
+        kv = int(rng.integers(2_000, 3_000_000))
+        pf = float(rng.uniform(1e9, 1.5e12))
+        if with_pure and i % 9 == 0:
+            pf = 0.0
+        if with_pure and i % 9 == 1:
+            kv = 0
+        dec, pre = 26.0 + 6.1e-4 * kv, 34.0 + 9.9e-10 * pf
+        lat = dec if pf == 0.0 else pre if kv == 0 else max(dec, pre)
+        lat = float(np.float32(lat * (1.0 + 0.04 * rng.standard_normal())))
+        r = ps.ps_grid_row()
+        r.token_batch, r.kv_tokens, r.prefill_flops, r.latency_us = b, kv, pf, lat
+        rows.append(r)
+        plain.append((b, kv, pf, lat))
+    return rows, plain
+
+
+def test_overlap_table_matches_the_oracle():
+    rng = np.random.default_rng(31)
+    for n, with_pure in ((648, True), (300, False), (40, True), (3, False)):
+        rows, plain = overlap_grid_rows(rng, n, with_pure)
+        t = S.ps_table_build_overlap(rows)
+        try:
+            want = so.table_build_overlap(plain)
+            b, base, s, q = S.ps_table_get_lines(t)
+            a_d, a_p = S.ps_table_get_overlap(t)
+            assert b.tolist() == [ln[0] for ln in want]
+            for i, ln in enumerate(want):
+                got = (base[i], a_d[i], s[i], a_p[i], q[i])
+                assert got[0] == 0.0 and all(abs(g - w) <= 1e-9 * max(1e-12, abs(w)) for g, w in zip(got, ln[1:]))
+            lines = list(zip(b.tolist(), base.tolist(), a_d.tolist(), s.tolist(), a_p.tolist(), q.tolist()))
+            for _ in range(1000):
+                tb, kv, pf = int(rng.integers(1, 4000)), int(rng.integers(0, 5_000_000)), float(rng.uniform(0, 2e12))
+                if rng.random() < 0.1:
+                    pf = 0.0
+                if rng.random() < 0.1:
+                    kv = 0
+                assert close(S.ps_table_predict(t, tb, kv, pf), so.table_predict(lines, tb, kv, pf))
+            # the batch term, the scaling and the admission test act on this form as on a sum table
+            S.ps_table_add_batch_term(t, [64, 512, 4096], [30.0, 150.0, 900.0])
+            S.ps_table_scale(t, 32.0)
+            more = so.table_scale(so.table_add_batch_term(lines, [(64, 30.0), (512, 150.0), (4096, 900.0)]), 32.0)
+            for tb, kv, pf in ((72, 100_000, 0.0), (500, 762_000, 1.2e11), (3000, 0, 4e11), (1, 5, 1.0)):
+                assert close(S.ps_table_predict(t, tb, kv, pf), so.table_predict(more, tb, kv, pf))
+            kv_len, rem = rng.integers(1, 9000, 64).astype(np.int32), rng.integers(1, 500, 64).astype(np.int32)
+            for tpot in (2e4, 6e4, 2e5):
+                got = S.ps_admit(t, kv_len, rem, 700, 300, 512, 4000, 8e10, tpot)
+                ok, pred, peak = so.admit(more, kv_len.tolist(), rem.tolist(), 700, 300, 512, 4000, 8e10, tpot)
+                assert bool(got[0]) == ok and close(got[1], pred) and got[2] == peak
+        finally:
+            S.ps_table_free(t)
+    # a sweep whose chunks never matter: the prefill side stays empty and keeps the start's values, slope not below 0
+    plain = [(96 + 32 * (i % 3), int(kv), float(pf), float(np.float32(30.0 + 6e-4 * kv - 2e-9 * pf + rng.normal(0, 0.5))))
+             for i, (kv, pf) in enumerate(zip(rng.integers(50_000, 900_000, 60), rng.uniform(1e8, 4e9, 60)))]
+    rows = []
+    for b, kv, pf, lat in plain:
+        r = ps.ps_grid_row()
+        r.token_batch, r.kv_tokens, r.prefill_flops, r.latency_us = b, kv, pf, lat
+        rows.append(r)
+    t = S.ps_table_build_overlap(rows)
+    want = so.table_build_overlap(plain)
+    _, _, s, q = S.ps_table_get_lines(t)
+    a_d, a_p = S.ps_table_get_overlap(t)
+    assert q[0] == 0.0 and want[0][5] == 0.0 and s[0] > 0
+    assert all(abs(g - w) <= 1e-9 * max(1e-12, abs(w)) for g, w in zip((a_d[0], s[0], a_p[0]), (want[0][2], want[0][3], want[0][4])))
+    S.ps_table_free(t)
+    t = S.ps_table_from_lines([5], [1.0], [0.1])
+    assert S.ps_table_get_overlap(t) is None
+    S.ps_table_free(t)
+    r = ps.ps_grid_row()
+    r.token_batch, r.kv_tokens, r.latency_us = 8, -1, 1.0
+    with pytest.raises(ps.PsError):
+        S.ps_table_build_overlap([r])
+
+
 def test_table_rejects_bad_input():
     with pytest.raises(ps.PsError):
         S.ps_table_from_lines([10, 10], [1.0, 2.0], [0.1, 0.1])  # duplicate batch size
