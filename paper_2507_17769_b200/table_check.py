@@ -12,7 +12,7 @@
 3. The host cost of the admission test (ps_admit) and of the chunk prediction (ps_chunk_predict) for an instance
    with 256 running requests, in decisions per second through this binding.
 4. With --iteration: the whole-iteration table of the paper's model T_iter = GEMM(B) + decode attention + prefill
-   attention (section 3.4) for an 8B-class decoder (32 layers, hidden 4096, 32 q / 8 kv heads of 128, FFN 14336): the
+   attention (section 3.4; the two attention terms in the overlap form) for an 8B-class decoder (32 layers, hidden 4096, 32 q / 8 kv heads of 128, FFN 14336): the
    sweep is repeated with the KV append inside the timed region, the linear layers' time at each of the table's batch
    sizes is measured with library GEMMs (torch.matmul, bf16; weights of four layers in rotation so that none is found
    in L2) and added with ps_table_add_batch_term, and everything is scaled to 32 layers with ps_table_scale.
@@ -105,7 +105,7 @@ def layer_gemm_us(batches, reps=20):
 
 def iteration_table(shape, grid, seeds, warmup, iters):
     rows = B.ps_profile_grid(shape, *grid, seeds, warmup, iters, 3000, include_kv_write=True)
-    table = S.ps_table_build(rows)
+    table = S.ps_table_build_overlap(rows)  # the form that predicts held-out batches best; its base takes GEMM(B)
     b, _, _, _ = S.ps_table_get_lines(table)
     gemm = layer_gemm_us(b.tolist())
     S.ps_table_add_batch_term(table, b, gemm)
