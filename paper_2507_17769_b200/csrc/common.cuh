@@ -241,6 +241,11 @@ __device__ __forceinline__ void bulk_g2s_hint(uint32_t dst, const void* src, uin
         "l"(src), "r"(bytes), "r"(bar), "l"(policy)
         : "memory");
 }
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
 __device__ __forceinline__ uint64_t l2_policy_evict_first() {
     uint64_t p;
     asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));

@@ -27,9 +27,18 @@ constexpr int kDecodeMinPagesLo = 4, kDecodeMinPagesHi = 8, kDecodePiecesPerRow 
 constexpr int kPrefillKeyTile = 128;    // keys per tensor-core tile
 // Measured on B200 (decode: bandwidth against the number of SMs the kernel runs on; prefill: time of one
 // key-tile step of a q tile pair), used to split the SMs of a mixed batch between the two kernels.
-constexpr double kDecodePeakBytesPerSec = 6.7e12;
-constexpr double kDecodeSharedPeakBytesPerSec = 6.0e12;  // decode rows beside a running prefill kernel
-constexpr double kDecodeBytesPerSecPerSm = 115e9;
+#ifndef PS_DECODE_PEAK
+#define PS_DECODE_PEAK 6.7e12
+#endif
+#ifndef PS_DECODE_SHARED_PEAK
+#define PS_DECODE_SHARED_PEAK 6.0e12
+#endif
+#ifndef PS_DECODE_PER_SM
+#define PS_DECODE_PER_SM 115e9
+#endif
+constexpr double kDecodePeakBytesPerSec = PS_DECODE_PEAK;
+constexpr double kDecodeSharedPeakBytesPerSec = PS_DECODE_SHARED_PEAK;  // decode rows beside a running prefill kernel
+constexpr double kDecodeBytesPerSecPerSm = PS_DECODE_PER_SM;
 constexpr double kDecodeAloneBytesPerSecPerSm = 135e9;  // per SM with the memory system to itself
 constexpr double kPrefillStepSec = 2.5e-6;
 constexpr double kKernelFloorSec = 12e-6;
