@@ -18,7 +18,10 @@ namespace ps {
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-constexpr int kDecodeUnitsPerWarp = 1;  // work units per resident warp (measured: 1 beats 2 and 3 on the decode-only batch)
+#ifndef PS_DECODE_UNITS_PER_WARP
+#define PS_DECODE_UNITS_PER_WARP 1
+#endif
+constexpr int kDecodeUnitsPerWarp = PS_DECODE_UNITS_PER_WARP;  // work units per resident warp (measured: 1 beats 2 and 3 on the decode-only batch)
 // Smallest decode unit (pages) of a batch too small to give every warp its share: between 4 and 8, so that the
 // longest row is cut into about 16 pieces at most.  Finer cuts spread a small batch over more warps (64 rows of
 // 64 tokens: 13 us instead of 20; 8 rows of 512: 16 instead of 23), but every further piece of a row is one more
