@@ -123,7 +123,13 @@ ps_status ps_kv_status(ps_kv *kv, void *stream);
 /*
  * Partition one batch into work items.  Rows with q_len == 1 are decode rows
  * (memory-bound KV streaming, section 2.2); rows with q_len > 1 are prefill
- * chunks (dense contraction, section 3.4).  Long contexts are cut into KV
+ * chunks (dense contraction, section 3.4).  A chunk of at most 8 tokens whose
+ * context is short enough to re-read (q_len * kv_len * bytes per token <= 32
+ * MB) is run as q_len decode rows instead -- token i as a row that sees
+ * prior + i + 1 keys of the same sequence -- in batches whose decode rows
+ * hold at most 128 MB of K/V and whose plan does not force prefill segments:
+ * there the prefill kernel's launch costs more than the re-reads.  Its items
+ * then appear among the decode items.  Long contexts are cut into KV
  * segments whose partial results are combined afterwards (decode rows inside
  * the decode kernel, prefill items by a merge kernel).  Host arrays
  * prior_host / q_len_host have n entries and are read before the call returns.

@@ -46,6 +46,21 @@ constexpr double kDecodeAloneBytesPerSecPerSm = 135e9;  // per SM with the memor
 constexpr double kPrefillStepSec = 2.5e-6;
 constexpr double kKernelFloorSec = 12e-6;
 
+// A chunk of a few tokens runs as that many decode rows (token i of the chunk is a row that sees prior + i + 1 keys
+// of the same sequence) instead of bringing in the prefill kernel for one small item: its launch and pipeline fill
+// cost more than re-reading a short context a few times.  Bounded by the bytes the rows re-read, and only in batches
+// whose decode rows are few: beside a long decode kernel the prefill kernel of a small chunk is hidden anyway.
+// (measured: a 2-token chunk on 2048 tokens beside 8 decode rows of 512: 23.8 us instead of 29.8; 8 tokens on 900
+// alone 16.4 instead of 22.6; 4 tokens on 1500 beside 128 rows of 2048 would be 169 instead of 165)
+constexpr int kTinyChunkTokens = 8;
+constexpr double kTinyChunkBytes = 32e6;
+constexpr double kTinyChunkMaxDecodeBytes = 128e6;
+static inline bool runs_as_decode(const ps_shape& sh, bool tiny_as_rows, int prior, int q_len) {
+    if (q_len == 1) return true;
+    if (!tiny_as_rows || q_len > kTinyChunkTokens) return false;
+    return (double)q_len * ((double)prior + q_len) * 2.0 * sh.n_kv_heads * sh.head_dim * 2.0 <= kTinyChunkBytes;
+}
+
 }  // namespace ps
 
 using namespace ps;
@@ -58,6 +73,7 @@ struct ps_plan {
     // (tensor-bound) run side by side on disjoint sets of SMs
     int32_t dec_sms = 0, pf_sms = 0;
     bool concurrent = false;
+    bool tiny_as_rows = false;  // this batch runs its chunks of a few tokens as decode rows
     std::vector<DecodePiece> pieces;
     std::vector<DecodeUnit> units;
     std::vector<PrefillItem> prefill;
@@ -106,11 +122,12 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
     const int Hkv = pl->shape.n_kv_heads, G = pl->shape.n_q_heads / Hkv;
     int64_t total_pages = 0, longest = 0;
     for (int r = 0; r < pl->n; ++r)
-        if (q_len[r] == 1) {
-            const int64_t pages = (prior[r] + 1 + kPage - 1) / kPage;
-            total_pages += pages * Hkv;
-            longest = std::max(longest, pages);
-        }
+        if (runs_as_decode(pl->shape, pl->tiny_as_rows, prior[r], q_len[r]))
+            for (int i = 0; i < q_len[r]; ++i) {
+                const int64_t pages = (prior[r] + i + 1 + kPage - 1) / kPage;
+                total_pages += pages * Hkv;
+                longest = std::max(longest, pages);
+            }
     if (total_pages == 0) {
         pl->pieces.clear();
         pl->units.clear();
@@ -130,7 +147,7 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
     // Upper bounds on the counts (a piece ends where its row or its unit ends), so that the lists are filled
     // in place and trimmed once.
     int64_t n_rows = 0;
-    for (int r = 0; r < pl->n; ++r) n_rows += q_len[r] == 1 ? Hkv : 0;
+    for (int r = 0; r < pl->n; ++r) n_rows += runs_as_decode(pl->shape, pl->tiny_as_rows, prior[r], q_len[r]) ? (int64_t)q_len[r] * Hkv : 0;
     const size_t max_units = (size_t)((total_pages + per_unit - 1) / per_unit);
     pl->pieces.resize((size_t)n_rows + max_units);
     pl->units.resize(max_units);
@@ -142,10 +159,11 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
     int64_t slots = *n_slots;
     int64_t room = 0;  // pages the open unit can still take
     for (int r = 0; r < pl->n; ++r) {
-        if (q_len[r] != 1) continue;
-        const int kv_len = prior[r] + 1;
+        if (!runs_as_decode(pl->shape, pl->tiny_as_rows, prior[r], q_len[r])) continue;
+        for (int i = 0; i < q_len[r]; ++i) {  // one row per new token (a decode request has one)
+        const int kv_len = prior[r] + i + 1;
         const int pages = (kv_len + kPage - 1) / kPage;
-        const int32_t q_tok = q_start[r];
+        const int32_t q_tok = q_start[r] + i;
         for (int g = 0; g < Hkv; ++g) {
             const int32_t first_piece = n_pieces;
             int pg = 0;
@@ -180,6 +198,7 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
                 slots += (int64_t)cnt * G;
             }
         }
+        }
     }
     if (n_units > 0) units[n_units - 1].piece_end = n_pieces;
     pl->pieces.resize((size_t)n_pieces);
@@ -206,11 +225,11 @@ static void plan_prefill(ps_plan* pl, const int32_t* prior, const int32_t* q_len
     std::vector<Tile> tiles;
     size_t n_tiles = 0;
     for (int r = 0; r < pl->n; ++r)
-        if (q_len[r] > 1) n_tiles += (size_t)((q_len[r] + tile_tok - 1) / tile_tok) * Hkv;
+        if (!runs_as_decode(pl->shape, pl->tiny_as_rows, prior[r], q_len[r])) n_tiles += (size_t)((q_len[r] + tile_tok - 1) / tile_tok) * Hkv;
     tiles.reserve(n_tiles);
     int64_t total_key_tiles = 0;
     for (int r = 0; r < pl->n; ++r) {
-        if (q_len[r] <= 1) continue;
+        if (runs_as_decode(pl->shape, pl->tiny_as_rows, prior[r], q_len[r])) continue;
         for (int g = 0; g < Hkv; ++g)
             for (int t0 = 0; t0 < q_len[r]; t0 += tile_tok) {
                 const int n_tok = std::min(tile_tok, q_len[r] - t0);
@@ -432,14 +451,22 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     pl->decode_merge_rows = 0;
     pl->prior.assign(prior_host, prior_host + n);
     pl->info = ps_plan_info{};
+    {
+        double true_dec_bytes = 0;
+        for (int r = 0; r < n; ++r)
+            if (q_len_host[r] == 1) true_dec_bytes += ((double)prior_host[r] + 1.0) * 2.0 * shape->n_kv_heads * shape->head_dim * 2.0;
+        // (forced prefill segments: the caller wants every chunk on the prefill kernel)
+        pl->tiny_as_rows = !(opts && opts->prefill_segment_tokens > 0) && true_dec_bytes <= kTinyChunkMaxDecodeBytes;
+    }
     // ---- split the SMs between the two kernels of a mixed batch ----
     {
         double dec_bytes = 0, pf_steps = 0;  // KV bytes the decode rows stream; key-tile steps of the prefill items
         const int G = shape->n_q_heads / shape->n_kv_heads;
         const int tile_tok = kPrefillRowsPerItem / G;
         for (int r = 0; r < n; ++r) {
-            if (q_len_host[r] == 1) {
-                dec_bytes += ((double)prior_host[r] + 1.0) * 2.0 * shape->n_kv_heads * shape->head_dim * 2.0;
+            if (runs_as_decode(*shape, pl->tiny_as_rows, prior_host[r], q_len_host[r])) {
+                for (int i = 0; i < q_len_host[r]; ++i)
+                    dec_bytes += ((double)prior_host[r] + i + 1.0) * 2.0 * shape->n_kv_heads * shape->head_dim * 2.0;
             } else {
                 for (int t0 = 0; t0 < q_len_host[r]; t0 += tile_tok) {
                     const int n_tok = std::min(tile_tok, q_len_host[r] - t0);
@@ -616,7 +643,7 @@ ps_status ps_plan_get_items(const ps_plan* pl, int32_t* decode_items_out, int64_
             o[4] = pc.q_tok;
             o[5] = 1;
             o[6] = pc.part_slot;
-            o[7] = pl->prior[pc.req];
+            o[7] = pc.kv_len - 1;  // the row's own position
         }
     }
     if (prefill_items_out) {

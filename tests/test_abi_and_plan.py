@@ -57,38 +57,44 @@ def coverage_check(batch, plan):
     G = s.group
     dec, pre = ps.ps_plan_get_items(plan)
     q_start = batch.q_start
-    # decode: per (req, kv head) the pieces tile [0, kv_len) in order
+    # decode: per (req, new token, kv head) the pieces tile [0, keys the token sees) in order; a decode request has
+    # one new token, a chunk of a few tokens may run as that many rows
     seen = {}
     for it in dec:
         r, g, k0, k1, qt, nt, slot, fp = it.tolist()
-        assert batch.q_len[r] == 1 and nt == 1 and qt == q_start[r] and fp == batch.prior[r]
-        assert k0 % 16 == 0 and k0 < k1 <= batch.kv_len[r]
-        seen.setdefault((r, g), []).append((k0, k1, slot))
+        i = qt - q_start[r]
+        assert nt == 1 and 0 <= i < batch.q_len[r] and fp == batch.prior[r] + i
+        assert k0 % 16 == 0 and k0 < k1 <= batch.prior[r] + i + 1
+        seen.setdefault((r, i, g), []).append((k0, k1, slot))
+    as_decode = {r for r, _, _ in seen}
     for r in range(batch.n):
-        if batch.q_len[r] != 1:
+        if batch.q_len[r] == 1:
+            assert r in as_decode
+        if r not in as_decode:
             continue
-        for g in range(s.n_kv_heads):
-            segs = sorted(seen[(r, g)])
-            assert segs[0][0] == 0 and segs[-1][1] == batch.kv_len[r]
-            for a, b in zip(segs[:-1], segs[1:]):
-                assert a[1] == b[0]
-            slots = [x[2] for x in segs]
-            if len(segs) == 1:
-                assert slots == [-1]
-            else:
-                assert all(x >= 0 for x in slots) and [x - slots[0] for x in slots] == [i * G for i in range(len(slots))]
+        for i in range(int(batch.q_len[r])):
+            for g in range(s.n_kv_heads):
+                segs = sorted(seen[(r, i, g)])
+                assert segs[0][0] == 0 and segs[-1][1] == batch.prior[r] + i + 1
+                for a, b in zip(segs[:-1], segs[1:]):
+                    assert a[1] == b[0]
+                slots = [x[2] for x in segs]
+                if len(segs) == 1:
+                    assert slots == [-1]
+                else:
+                    assert all(x >= 0 for x in slots) and [x - slots[0] for x in slots] == [k * G for k in range(len(slots))]
     # prefill: per (req, kv head, tile) the segments tile [0, first_pos + n_tok)
     tiles = {}
     for it in pre:
         r, g, k0, k1, qt, nt, slot, fp = it.tolist()
-        assert batch.q_len[r] > 1 and k0 % 128 == 0 and k0 < k1
+        assert batch.q_len[r] > 1 and r not in as_decode and k0 % 128 == 0 and k0 < k1
         tok0 = qt - q_start[r]
         assert fp == batch.prior[r] + tok0 and 1 <= nt <= 256 // G and tok0 % (256 // G) == 0
         assert k1 <= fp + nt
         tiles.setdefault((r, g, tok0, nt), []).append((k0, k1, slot))
     for r in range(batch.n):
         c = int(batch.q_len[r])
-        if c <= 1:
+        if r in as_decode:
             continue
         tt = 256 // G
         for g in range(s.n_kv_heads):
@@ -109,7 +115,7 @@ def coverage_check(batch, plan):
     # partial slots of different groups never overlap
     info = ps.ps_plan_get_info(plan)
     used = np.zeros(info.n_partial_slots, dtype=np.int32)
-    for (r, g), segs in seen.items():
+    for _, segs in seen.items():
         for k0, k1, slot in segs:
             if slot >= 0:
                 used[slot : slot + G] += 1
@@ -134,6 +140,50 @@ def test_partition_covers_every_row_and_key_once(make, kw):
         info = coverage_check(batch, plan)
         assert info.total_q_tokens == batch.total_q
         assert ws >= 256 + info.n_partial_slots * (batch.shape.head_dim + 1) * 4
+    finally:
+        ps.ps_plan_free(plan)
+
+
+def test_chunks_of_a_few_tokens_run_as_decode_rows():
+    """Up to 8 new tokens on a context short enough to re-read: one decode row per token, no prefill item.  Longer
+    chunks, long contexts and plans with forced prefill segments keep the prefill kernel."""
+    shape = gen.SHAPE_8B
+    b = gen.make_batch(shape, 5, [2048, 0, 100, 511, 7, 300, 60000], [2, 8, 1, 5, 9, 1, 4])
+    plan, _ = ps.ps_attn_plan(ps.make_shape(32, 8, 128), b.prior, b.q_len, b.max_pages, opts(), None)
+    try:
+        info = coverage_check(b, plan)
+        dec, pre = ps.ps_plan_get_items(plan)
+        assert set(pre[:, 0].tolist()) == {4, 6}  # the 9-token chunk, and 4 tokens on 60 000 (a 1 GB re-read)
+        assert set(dec[:, 0].tolist()) == {0, 1, 2, 3, 5}
+        rows = {(r, qt) for r, qt in zip(dec[:, 0].tolist(), dec[:, 4].tolist())}
+        assert len(rows) == 2 + 8 + 1 + 5 + 1
+        assert info.n_prefill_items == len(pre) > 0
+    finally:
+        ps.ps_plan_free(plan)
+    plan, _ = ps.ps_attn_plan(ps.make_shape(32, 8, 128), b.prior, b.q_len, b.max_pages, opts(pre=128), None)
+    try:
+        coverage_check(b, plan)
+        dec, pre = ps.ps_plan_get_items(plan)
+        assert set(dec[:, 0].tolist()) == {2, 5} and set(pre[:, 0].tolist()) == {0, 1, 3, 4, 6}
+    finally:
+        ps.ps_plan_free(plan)
+    # a batch of tiny chunks only launches the decode kernel alone
+    b = gen.make_batch(shape, 6, [2048, 10], [2, 3])
+    plan, _ = ps.ps_attn_plan(ps.make_shape(32, 8, 128), b.prior, b.q_len, b.max_pages, opts(), None)
+    try:
+        info = coverage_check(b, plan)
+        assert info.n_prefill_items == 0 and info.n_launches == 1 and info.decode_sms == info.prefill_sms == 148
+    finally:
+        ps.ps_plan_free(plan)
+
+
+    # beside many decode rows the chunk's prefill kernel is hidden: it stays a prefill item
+    b = gen.make_batch(shape, 7, [1500] + [2047] * 128, [4] + [1] * 128)
+    plan, _ = ps.ps_attn_plan(ps.make_shape(32, 8, 128), b.prior, b.q_len, b.max_pages, opts(), None)
+    try:
+        coverage_check(b, plan)
+        _, pre = ps.ps_plan_get_items(plan)
+        assert set(pre[:, 0].tolist()) == {0}
     finally:
         ps.ps_plan_free(plan)
 

@@ -107,6 +107,20 @@ def test_prefill_chunks(prior, c, shape):
     full_parity(b, what="prefill prior=%d c=%d" % (prior, c))
 
 
+@pytest.mark.parametrize("shape", [gen.SHAPE_8B, gen.Shape(8, 8, 64), gen.SHAPE_LARGE])
+def test_chunks_of_a_few_tokens_on_either_kernel(shape):
+    """Chunks of 2 to 8 tokens run as decode rows by default and on the prefill kernel when segments are forced;
+    both match the oracle."""
+    b = gen.make_batch(shape, 45, [0, 5, 127, 1000, 300, 1200, 64], [2, 3, 8, 2, 1, 5, 9])
+    (_, _), info, db, out_a, _ = full_parity(b, what="tiny chunks as decode rows")
+    _, pre = ps.ps_plan_get_items(db.pa._plan)
+    assert set(pre[:, 0].tolist()) == {6}  # only the 9-token chunk
+    (_, _), info, db, out_b, _ = full_parity(b, ps.ps_plan_opts(0, 128, 0), what="tiny chunks on the prefill kernel")
+    _, pre = ps.ps_plan_get_items(db.pa._plan)
+    assert set(pre[:, 0].tolist()) == {0, 1, 2, 3, 5, 6}
+    assert (out_a.float() - out_b.float()).abs().max().item() <= 1e-2
+
+
 @pytest.mark.parametrize("seg", [128, 256])
 def test_prefill_split_kv_and_merge(seg):
     b = gen.make_batch(gen.SHAPE_8B, 41, [700, 100], [40, 200])
