@@ -447,7 +447,7 @@ def run_ours(args):
             "roofline": roof,
             "kernels": extra,
         }
-        # ---- CPU baseline: the oracle as it stands, on this machine's host cores ----
+        # ---- CPU baseline: the oracle as it stands, on the host's cores ----
         if world == 1 and not args.no_cpu_baseline:
             reqs = oracle_sample(batch)
             dt, nbytes, threads = time_oracle(batch, reqs)
