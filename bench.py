@@ -55,7 +55,7 @@ def measured_peaks():
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel from one ncu capture (see
 # profiles/decode_kernel_config1.md), valid only for the kernel source it was taken on.
-NCU_TRAFFIC = {1: {"decode_cu_sha256_prefix": "740814e60edf27c5", "bytes_per_launch": 601.1e6}}
+NCU_TRAFFIC = {1: {"decode_cu_sha256_prefix": "740814e60edf27c5", "bytes_per_launch": 600.8e6}}
 
 
 def ncu_traffic(workload):
