@@ -160,7 +160,7 @@ typedef struct {
     int64_t n_partial_slots;   /* fp32 partial rows held in the workspace */
     int64_t total_q_tokens;
     int32_t n_launches;        /* kernels one ps_attn_run launches for this plan */
-    int32_t decode_sms;        /* SMs the decode kernel is sized for (alone: 7/8 of them, from where it streams fastest) */
+    int32_t decode_sms;        /* SMs the decode kernel is sized for */
     int32_t prefill_sms;       /* SMs the prefill kernel is sized for; in a mixed batch the two kernels run side by
                                   side on disjoint SMs when that is predicted to be faster (decode_sms + prefill_sms
                                   = all SMs), otherwise one after the other on all of them */

@@ -460,14 +460,13 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     }
     // ---- split the SMs between the two kernels of a mixed batch ----
     {
-        double dec_bytes = 0, pf_steps = 0, dec_rows = 0;  // KV bytes the decode rows stream; key-tile steps of the prefill items
+        double dec_bytes = 0, pf_steps = 0;  // KV bytes the decode rows stream; key-tile steps of the prefill items
         const int G = shape->n_q_heads / shape->n_kv_heads;
         const int tile_tok = kPrefillRowsPerItem / G;
         for (int r = 0; r < n; ++r) {
             if (runs_as_decode(*shape, pl->tiny_as_rows, prior_host[r], q_len_host[r])) {
                 for (int i = 0; i < q_len_host[r]; ++i)
                     dec_bytes += ((double)prior_host[r] + i + 1.0) * 2.0 * shape->n_kv_heads * shape->head_dim * 2.0;
-                dec_rows += q_len_host[r];
             } else {
                 for (int t0 = 0; t0 < q_len_host[r]; t0 += tile_tok) {
                     const int n_tok = std::min(tile_tok, q_len_host[r] - t0);
@@ -476,14 +475,6 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
             }
         }
         pl->dec_sms = pl->pf_sms = pl->num_sms;
-        // Rows of a few hundred tokens and more stream fastest from about 7/8 of the SMs: with all of them the memory
-        // system is oversubscribed (measured on 148 SMs, us per run at 148 / 132 / 128 / 124 CTAs: 64 sequences of
-        // U[512, 4096) 98.0 / 95.4 / 96.4 / 95.6; 512 sequences 469 / 454 / 456 / 455; 256 long sequences 2745 / 2653
-        // / 2640 / 2646 = 7.19 TB/s; 136 and 140 CTAs are slower than either neighbour).  Batches of short rows are
-        // bound by per-row work and keep every SM (4096 rows of U[1, 200) tokens: 301 us on 148, 308 on 128); small
-        // batches launch fewer CTAs than either count anyway.
-        if (pl->num_sms >= 64 && dec_rows > 0 && dec_bytes >= dec_rows * 256.0 * 2.0 * shape->n_kv_heads * shape->head_dim * 2.0)
-            pl->dec_sms = pl->num_sms * 7 / 8 / 4 * 4;
         pl->concurrent = false;
         if (dec_bytes > 0 && pf_steps > 0 && pl->num_sms >= 16) {
             // time models (seconds): decode = bytes / min(side-by-side peak, n * per-SM rate); prefill = steps * step time / m

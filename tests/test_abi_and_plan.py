@@ -172,7 +172,7 @@ def test_chunks_of_a_few_tokens_run_as_decode_rows():
     plan, _ = ps.ps_attn_plan(ps.make_shape(32, 8, 128), b.prior, b.q_len, b.max_pages, opts(), None)
     try:
         info = coverage_check(b, plan)
-        assert info.n_prefill_items == 0 and info.n_launches == 1 and (info.decode_sms, info.prefill_sms) == (128, 148)
+        assert info.n_prefill_items == 0 and info.n_launches == 1 and info.decode_sms == info.prefill_sms == 148
     finally:
         ps.ps_plan_free(plan)
 
@@ -207,17 +207,6 @@ def test_partition_ignores_page_ids_and_replans_in_place():
     ps.ps_plan_free(plan2)
 
 
-def test_batches_of_short_decode_rows_keep_every_sm():
-    sh = ps.make_shape(32, 8, 128)
-    rng = np.random.default_rng(9)
-    for lo, hi, want in ((1, 200, 148), (200, 600, 128), (16, 2048, 128)):
-        ctx = rng.integers(lo, hi, 1024)
-        b = gen.make_batch(gen.SHAPE_8B, 9, ctx - 1, np.ones(1024, dtype=np.int32))
-        plan, _ = ps.ps_attn_plan(sh, b.prior, b.q_len, b.max_pages, opts())
-        assert ps.ps_plan_get_info(plan).decode_sms == want
-        ps.ps_plan_free(plan)
-
-
 def test_decode_units_are_balanced():
     b = gen.config1()
     sh = ps.make_shape(32, 8, 128)
@@ -225,7 +214,7 @@ def test_decode_units_are_balanced():
     info = ps.ps_plan_get_info(plan)
     total_pages = int(((b.kv_len + 15) // 16).sum()) * 8
     per_unit = info.decode_segment_tokens // 16
-    assert per_unit == max(8, -(-total_pages // (info.decode_sms * 12))) and info.decode_sms == 128  # one unit per resident warp (12 warps per SM)
+    assert per_unit == max(8, -(-total_pages // (148 * 12)))  # one unit per resident warp (12 warps per SM)
     # partial rows stay a small fraction of the KV stream
     assert info.n_partial_slots * 128 * 4 < 0.1 * b.decode_bytes()
     ps.ps_plan_free(plan)
@@ -240,8 +229,8 @@ def test_mixed_batches_split_the_sms_and_single_class_batches_do_not():
         info = ps.ps_plan_get_info(plan)
         if mixed:
             assert info.decode_sms + info.prefill_sms == 148 and info.decode_sms >= 8 and info.prefill_sms >= 8
-        else:  # no split: a kernel has the GPU to itself; decode rows of some length stream fastest from 7/8 of the SMs
-            assert info.decode_sms == (128 if (b.q_len == 1).any() else 148) and info.prefill_sms == 148
+        else:
+            assert info.decode_sms == 148 and info.prefill_sms == 148
         coverage_check(b, plan)
         ps.ps_plan_free(plan)
     big = gen.config4()
