@@ -202,6 +202,12 @@ ps_status ps_plan_get_items(const ps_plan *plan, int32_t *decode_items_out, int6
  * kernel), and is joined back into `stream` before the call's work is
  * complete in stream order.  Consecutive runs of one plan must be issued to the
  * same stream, or be ordered by the caller: they share the partial buffers.
+ * The call may be made while `stream` is being captured into a CUDA graph:
+ * the upload then becomes a node of the graph on `stream` (each replay copies
+ * the plan's staging image again) and the graph replays this plan, with these
+ * pointers, as often as wanted.  The graph belongs to the plan as it was
+ * captured: after ps_attn_plan on the same plan object capture again, and do
+ * not re-plan or free the plan while a replay is in flight.
  * Returns host-detectable errors only (PS_ERR_INVALID, PS_ERR_WORKSPACE,
  * PS_ERR_CUDA); errors seen on the device are read with ps_plan_status.
  */

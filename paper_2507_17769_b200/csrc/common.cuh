@@ -23,9 +23,11 @@ void clear_error();
 #define PS_CUDA_TRY(expr)                                                                     \
     do {                                                                                      \
         cudaError_t e__ = (expr);                                                             \
-        if (e__ != cudaSuccess)                                                               \
+        if (e__ != cudaSuccess) {                                                             \
+            (void)cudaGetLastError(); /* reported here: do not leave it for an unrelated later call */ \
             return ps::fail(PS_ERR_CUDA, "%s failed: %s (%s:%d)", #expr, cudaGetErrorString(e__), \
                             __FILE__, __LINE__);                                              \
+        }                                                                                     \
     } while (0)
 
 ps_status check_shape(const ps_shape* s);

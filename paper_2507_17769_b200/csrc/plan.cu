@@ -667,7 +667,17 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     char* const ws_base = (char*)workspace_dev;
     const int slot = (int)(pl->run_no++ & 1u);
     char* ws = ws_base + (size_t)slot * pl->image_bytes;  // this run's image slot; partials are addressed from ws_base
-    if (pl->copy_stream) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    PS_CUDA_TRY(cudaStreamIsCapturing(s, &cap));
+    const bool capturing = cap != cudaStreamCaptureStatusNone;
+    if (capturing) {
+        // Inside a stream capture the upload is a node of the graph on the caller's stream: every replay copies the
+        // staging image as it then stands.  Nothing recorded here may be waited for by a later call outside the
+        // capture, so the slot bookkeeping starts afresh.
+        PS_CUDA_TRY(cudaMemcpyAsync(ws, pl->pinned, pl->image_bytes, cudaMemcpyHostToDevice, s));
+        pl->done_valid[0] = pl->done_valid[1] = false;
+        pl->last_ws = workspace_dev;
+    } else if (pl->copy_stream) {
         cudaStream_t cs = pl->copy_stream;
         if (pl->last_ws == workspace_dev && pl->done_valid[slot]) {
             // same workspace as before: the slot is free once the run two calls ago has finished
@@ -720,7 +730,7 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     a.w.n_prefill_ctas = pl->prefill_cta_start.empty() ? 0 : (int32_t)pl->prefill_cta_start.size() - 1;
 
     // events per recorded run: prefill begin/end, decode begin/end, merge begin/end
-    const bool rec = pl->timing && (size_t)(pl->timed_runs + 1) * 6 <= pl->tev.size();
+    const bool rec = !capturing && pl->timing && (size_t)(pl->timed_runs + 1) * 6 <= pl->tev.size();
     cudaEvent_t* ev = rec ? &pl->tev[(size_t)pl->timed_runs * 6] : nullptr;
     ps_status st = PS_OK;
     bool merged = false;  // the merge kernel has been launched already
@@ -777,7 +787,7 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
         if (rec) cudaEventRecord(ev[5], s);
     }
     if (rec) ++pl->timed_runs;
-    if (pl->copy_stream && st == PS_OK) {
+    if (pl->copy_stream && st == PS_OK && !capturing) {
         PS_CUDA_TRY(cudaEventRecord(pl->ev_done[slot], s));
         pl->done_valid[slot] = true;
     }
