@@ -5,10 +5,13 @@
 
 A step is one pass of the whole path over one synthetic batch: host work
 partition (ps_attn_plan), then ps_attn_run (work-list upload, prefill, decode
-and merge kernels).  The default workload is the decode-only 8B-class batch
-(64 sequences, contexts uniform on [512, 4096], about 0.6 GB of KV, larger than
-L2); the headline value is the KV bytes the decode rows must stream divided by
-the step time.  With N > 1 (torchrun) every rank runs its own batch of the same
+and merge kernels).  The default workload is the largest single-GPU batch:
+256 decode sequences with contexts uniform on [4096, 32768] beside two
+2048-token prefill chunks on 16 k - 30 k prior tokens, 64 q / 8 kv heads (about
+19 GB of KV; the two kernels run side by side).  The headline value is the KV
+bytes the decode rows must stream divided by the step time; the prefill rows'
+TFLOP/s over the same step, the roofline fraction of the step and of each
+kernel, and the CPU oracle's rates on a bounded sample are in the same line.  With N > 1 (torchrun) every rank runs its own batch of the same
 law (weak scaling, no data-path collective); the step time is the maximum over
 ranks and the value the sum of all ranks' bytes over that time.  With
 ``--shard heads`` the ranks instead split ONE batch by KV head (rank k takes kv
@@ -53,25 +56,19 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the decode kernel from one ncu capture (see
-# profiles/decode_kernel_config1.md), valid only for the kernel source it was taken on.
-NCU_TRAFFIC = {1: {"decode_cu_sha256_prefix": "740814e60edf27c5", "bytes_per_launch": 600.8e6}}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch, as a multiple of the launch's algorithmic bytes, from the
+# ncu captures summarised under profiles/ (small cases of the same kernels; DRAM traffic of both kernels grows in
+# proportion to the KV a launch reads, so a full launch is the ratio times its algorithmic bytes).  The decode
+# kernel's algorithmic bytes are the KV it streams; for the prefill kernel the ratio is per KV byte of its chunks'
+# sequences (its K/V tiles are re-read from L2, not from DRAM).  Re-captured whenever a kernel changes.
+NCU_TRAFFIC_RATIO = {"decode_kernel": 1.012}
+NCU_TRAFFIC_SOURCE = "profiles/decode_kernel_config1.md"
 
 
-def ncu_traffic(workload):
-    """Measured DRAM traffic per launch, or None if the kernel changed since the counters were taken."""
-    import hashlib
-
-    rec = NCU_TRAFFIC.get(workload)
-    if rec is None:
-        return None
-    src = os.path.join(ROOT, "paper_2507_17769_b200", "csrc", "decode.cu")
-    try:
-        with open(src, "rb") as f:
-            digest = hashlib.sha256(f.read()).hexdigest()
-    except OSError:
-        return None
-    return rec["bytes_per_launch"] if digest.startswith(rec["decode_cu_sha256_prefix"]) else None
+def ncu_traffic(kernel, algorithmic_units):
+    """DRAM bytes per launch of ``kernel`` scaled from the committed capture, or None where no capture exists."""
+    ratio = NCU_TRAFFIC_RATIO.get(kernel)
+    return None if ratio is None else ratio * algorithmic_units
 
 
 class ClockSampler:
@@ -180,56 +177,140 @@ def shard_batch(make, seed, rank, world, shard):
     return gen.make_batch(part, seed, full.prior, full.q_len)
 
 
-def oracle_sample(batch, budget_flops=6e10):
-    """Decode requests of ``batch`` for the CPU oracle, bounded by an fp64 flop budget."""
+def oracle_sample(batch, dec_flops=4e10, pf_flops=8e10):
+    """A bounded sample of ``batch`` for the CPU oracle: decode requests from the front of the batch up to
+    ``dec_flops`` of fp64 work, and new-token rows spread evenly over every prefill chunk up to ``pf_flops``.
+    Returns (decode requests, {chunk request: row indices})."""
     s = batch.shape
-    cost = 4.0 * s.head_dim * s.n_q_heads * (batch.prior.astype(np.float64) + 1.0)
-    picked, tot = [], 0.0
+    phi = 4.0 * s.head_dim * s.n_q_heads
+    dec, tot = [], 0.0
     for r in range(batch.n):
         if batch.q_len[r] > 1:
-            continue  # decode rows carry the headline metric
-        if tot + cost[r] > budget_flops and picked:
+            continue
+        cost = phi * (float(batch.prior[r]) + 1.0)
+        if dec and tot + cost > dec_flops:
             break
-        picked.append(r)
-        tot += cost[r]
-    return picked
+        dec.append(r)
+        tot += cost
+    chunks = [r for r in range(batch.n) if batch.q_len[r] > 1]
+    rows = {}
+    for r in chunks:
+        per_row = phi * (float(batch.prior[r]) + 0.5 * float(batch.q_len[r]))
+        k = int(max(1, min(int(batch.q_len[r]), pf_flops / len(chunks) / per_row)))
+        rows[r] = sorted(set(np.linspace(0, int(batch.q_len[r]) - 1, k).astype(int).tolist()))
+    return dec, rows
 
 
-def time_oracle(batch, reqs):
-    """Seconds the oracle takes on the given requests (inputs built outside the timed part)."""
-    import oracle
+def sample_text(batch, dec, rows):
+    n_dec = int((batch.q_len == 1).sum())
+    txt = "%d of %d decode requests" % (len(dec), n_dec)
+    if rows:
+        txt += " + %d of %d chunk rows (evenly spaced over %d chunk%s)" % (
+            sum(len(v) for v in rows.values()), int(batch.q_len[batch.q_len > 1].sum()), len(rows), "s" if len(rows) > 1 else "")
+    return txt + "; the whole step's time is extrapolated from the two measured rates by algorithmic work"
+
+
+def host_bits(batch, r, device):
+    """K, V and Q bit patterns of request r on the host.  With a CUDA device they come from the input generator's
+    device twin (bit-identical to the numpy generator, which needs minutes for the large configs)."""
+    import torch
 
     s = batch.shape
-    ks, vs, qs = [], [], []
-    for r in reqs:
-        k, v = batch.kv_bits(r)
-        ks.append(k)
-        vs.append(v)
-        qs.append(gen.gen_q(batch.seed, r, int(batch.prior[r]), int(batch.prior[r] + batch.q_len[r]), s.n_q_heads, s.head_dim))
-    need = [(x.shape[0] + s.page_size - 1) // s.page_size for x in ks]
-    bt = np.full((len(reqs), max(need)), -1, dtype=np.int32)
-    off = 0
-    for a, c in enumerate(need):
-        bt[a, :c] = np.arange(off, off + c)
-        off += c
-    kp = oracle.plain_pool(ks, bt, off + 1, s.page_size)
-    vp = oracle.plain_pool(vs, bt, off + 1, s.page_size)
-    q = np.concatenate(qs)
-    args = (q, kp, vp, bt, batch.prior[reqs], batch.q_len[reqs], s.n_q_heads, s.n_kv_heads, s.head_dim, s.page_size)
-    t0 = time.perf_counter()
-    oracle.attn_paged(*args)
-    dt = time.perf_counter() - t0
-    nbytes = float((batch.kv_len[reqs][batch.q_len[reqs] == 1]).sum()) * s.kv_token_bytes
-    return dt, nbytes, oracle.num_threads()
+    lo, hi = int(batch.prior[r]), int(batch.kv_len[r])
+    if device is not None:
+        from workloads import gen_cuda
+
+        def bits(t):
+            return t.contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+        k, v = gen_cuda.gen_kv(batch.seed, r, 0, hi, s.n_kv_heads, s.head_dim, device)
+        return bits(k), bits(v), bits(gen_cuda.gen_q(batch.seed, r, lo, hi, s.n_q_heads, s.head_dim, device))
+    k, v = batch.kv_bits(r)
+    return k, v, gen.gen_q(batch.seed, r, lo, hi, s.n_q_heads, s.head_dim)
+
+
+class OracleSample:
+    """Inputs of a bounded sample, built once; ``time()`` runs the oracle on them and returns the two rates."""
+
+    def __init__(self, batch, dec, rows, device=None):
+        import oracle
+
+        self.batch, self.dec, self.rows = batch, dec, rows
+        s = batch.shape
+        self.parts = []
+        for reqs, row_sel in ((dec, None), (sorted(rows), rows)):
+            if not reqs:
+                self.parts.append(None)
+                continue
+            ks, vs, qs = [], [], []
+            for r in reqs:
+                k, v, q = host_bits(batch, r, device)
+                ks.append(k)
+                vs.append(v)
+                qs.append(q)
+            need = [(x.shape[0] + s.page_size - 1) // s.page_size for x in ks]
+            bt = np.full((len(reqs), max(need)), -1, dtype=np.int32)
+            off = 0
+            for a, c in enumerate(need):
+                bt[a, :c] = np.arange(off, off + c)
+                off += c
+            kp = oracle.plain_pool(ks, bt, off + 1, s.page_size)
+            vp = oracle.plain_pool(vs, bt, off + 1, s.page_size)
+            row_req, row_tok, work = [], [], 0.0
+            for a, r in enumerate(reqs):
+                for i in (range(int(batch.q_len[r])) if row_sel is None else row_sel[r]):
+                    row_req.append(a)
+                    row_tok.append(i)
+                    work += float(batch.prior[r]) + i + 1.0  # keys this row sees
+            self.parts.append((np.concatenate(qs), kp, vp, bt, batch.prior[reqs], batch.q_len[reqs], row_req, row_tok, work))
+
+    def time(self):
+        """(seconds on the decode sample, its KV bytes, seconds on the chunk-row sample, its flops, threads)."""
+        import oracle
+
+        s = self.batch.shape
+        res = []
+        for part in self.parts:
+            if part is None:
+                res.append((0.0, 0.0))
+                continue
+            q, kp, vp, bt, prior, q_len, row_req, row_tok, work = part
+            t0 = time.perf_counter()
+            oracle.attn_rows(q, kp, vp, bt, prior, q_len, s.n_q_heads, s.n_kv_heads, s.head_dim, s.page_size, row_req, row_tok)
+            res.append((time.perf_counter() - t0, work))
+        (dt_d, keys_d), (dt_p, keys_p) = res
+        return dt_d, keys_d * s.kv_token_bytes, dt_p, keys_p * 4.0 * s.head_dim * s.n_q_heads, oracle.num_threads()
+
+    def whole_step(self, dt_d, bytes_d, dt_p, flops_p):
+        """Seconds the oracle would need for the whole batch, from the two measured rates."""
+        full = 0.0
+        if bytes_d > 0:
+            full += float(self.batch.decode_bytes()) * dt_d / bytes_d
+        if flops_p > 0:
+            full += float(self.batch.prefill_flops()) * dt_p / flops_p
+        return full
+
+
+def cpu_baseline_record(batch, sample, timing):
+    dt_d, bytes_d, dt_p, flops_p, threads = timing
+    full = sample.whole_step(dt_d, bytes_d, dt_p, flops_p)
+    return {"value": float(batch.decode_bytes()) / full / 1e12, "unit": "TB/s", "cores": threads, "kind": "oracle",
+            "sample": sample_text(batch, sample.dec, sample.rows), "sample_seconds": dt_d + dt_p,
+            "whole_step_seconds_extrapolated": full,
+            "decode_TBps": bytes_d / dt_d / 1e12 if dt_d > 0 else None,
+            "prefill_TFLOPs": flops_p / dt_p / 1e12 if dt_p > 0 else None}
 
 
 def components_alone(pa, batch, db, out, steps, peaks):
-    """Decode rows alone and prefill rows alone (each on all SMs), for attribution in mixed batches."""
+    """Decode rows alone and prefill rows alone (each planned by itself on all SMs), for attribution in mixed batches.
+    Returns one record per row class for the roofline's kernel list."""
     import torch
+    import paper_2507_17769_b200 as ps
 
-    res = {}
+    res = []
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     q_start = batch.q_start
+    stream = torch.cuda.current_stream(db.q.device)
     for name, mask in (("decode", batch.q_len == 1), ("prefill", batch.q_len > 1)):
         idx = np.nonzero(mask)[0]
         rows = torch.from_numpy(idx).to(db.block_table.device)
@@ -252,17 +333,36 @@ def components_alone(pa, batch, db, out, steps, peaks):
             step()
         ev1.record()
         torch.cuda.synchronize()
-        ms = ev0.elapsed_time(ev1) / n
+        step_ms = ev0.elapsed_time(ev1) / n
+        ps.ps_plan_set_timing(pa._plan, n)
+        for _ in range(n):
+            step()
+        pre_ms, dec_ms, _, _ = ps.ps_plan_get_timing(pa._plan, stream.cuda_stream)
+        ps.ps_plan_set_timing(pa._plan, 0)
         if name == "decode":
-            res["decode_rows_alone_ms"] = ms
-            res["decode_rows_alone_TBps"] = float(batch.decode_bytes()) / (ms * 1e-3) / 1e12
+            res.append(kernel_record("decode_kernel", "decode rows alone on all SMs", dec_ms, float(batch.decode_bytes()), peaks,
+                                     step_ms=step_ms))
         else:
-            tf = float(batch.prefill_flops()) / (ms * 1e-3) / 1e12
-            res["prefill_rows_alone_ms"] = ms
-            res["prefill_rows_alone_TFLOPs"] = tf
-            res["prefill_rows_alone_frac_of_bf16_peak"] = tf / peaks["bf16_tflops"]
+            res.append(kernel_record("prefill_kernel", "prefill rows alone on all SMs", pre_ms, float(batch.prefill_flops()), peaks,
+                                     step_ms=step_ms))
     pa.plan(batch.prior, batch.q_len, batch.max_pages)  # back to the full batch
     return res
+
+
+def kernel_record(kernel, where, launch_ms, units, peaks, step_ms=None):
+    """One entry of the roofline's kernel list: algorithmic units of one launch over its CUDA-event duration."""
+    if kernel == "decode_kernel":
+        ach = units / (launch_ms * 1e-3) / 1e9 if launch_ms > 0 else 0.0
+        rec = {"kernel": kernel, "where": where, "bound": "hbm", "launch_ms": launch_ms, "algorithmic_bytes_per_launch": units,
+               "achieved": ach, "unit": "GB/s", "peak": peaks["hbm_gbs"], "frac": ach / peaks["hbm_gbs"]}
+    else:
+        ach = units / (launch_ms * 1e-3) / 1e12 if launch_ms > 0 else 0.0
+        rec = {"kernel": kernel, "where": where, "bound": "tensor", "launch_ms": launch_ms, "algorithmic_flops_per_launch": units,
+               "achieved": ach, "unit": "TFLOP/s", "peak": peaks["bf16_tflops"], "frac": ach / peaks["bf16_tflops"],
+               "peak_sustained": peaks["bf16_tflops_sustained"], "frac_of_sustained": ach / peaks["bf16_tflops_sustained"]}
+    if step_ms is not None:
+        rec["step_ms"] = step_ms
+    return rec
 
 
 def run_reference(args):
@@ -271,22 +371,33 @@ def run_reference(args):
         return 0
     desc, make, seed = WORKLOADS[args.workload]
     batch = make(seed)
-    reqs = oracle_sample(batch)
-    if args.warmup > 0:
-        time_oracle(batch, reqs[:2])
-    times, nbytes, threads = [], 0.0, 1
+    device = None
+    try:
+        import torch
+
+        if torch.cuda.is_available():
+            device = torch.device("cuda", 0)
+    except ImportError:
+        pass
+    dec, rows = oracle_sample(batch)
+    sample = OracleSample(batch, dec, rows, device)
+    for _ in range(min(args.warmup, 1)):
+        sample.time()
+    acc = None
     for _ in range(args.steps):
-        dt, nbytes, threads = time_oracle(batch, reqs)
-        times.append(dt)
-    ms = 1e3 * sum(times) / len(times)
-    value = nbytes / (ms * 1e-3) / 1e12
-    sample = "%d of %d decode requests (%.1f MB of KV) per step" % (len(reqs), batch.n, nbytes / 1e6)
+        t = sample.time()
+        acc = t if acc is None else tuple(a + b for a, b in zip(acc[:4], t[:4])) + (t[4],)
+    timing = tuple(x / args.steps for x in acc[:4]) + (acc[4],)
+    rec = cpu_baseline_record(batch, sample, timing)
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": "TB/s", "n_gpus": args.gpus, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f64", "data": "synthetic", "config": {"workload": desc, "sample": sample},
-        "cpu_baseline": {"value": value, "unit": "TB/s", "cores": threads, "kind": "oracle", "sample": sample},
-        "e2e": {"value": value, "unit": "TB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "impl": "reference", "metric": METRIC, "value": rec["value"], "unit": "TB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * rec["sample_seconds"], "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": desc, "sample": rec["sample"],
+                   "note": "a step is one oracle pass over the sample; value = the batch's decode KV bytes over the "
+                           "whole-step time extrapolated from the sample's rates"},
+        "cpu_baseline": rec,
+        "e2e": {"value": rec["value"], "unit": "TB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
     return 0
@@ -349,8 +460,9 @@ def run_ours(args):
         ev1.record(stream)
         barrier()
         local_ms = ev0.elapsed_time(ev1) / args.steps
-        # pass 2: the same steps again with events around every kernel launch, for the per-kernel
-        # durations of the roofline (kept out of pass 1: each extra event costs device time)
+        # pass 2: the same steps again with events around every kernel launch (on the stream each kernel is
+        # launched on), for the per-kernel durations of the roofline (kept out of pass 1: each extra event costs
+        # device time)
         n_kernel_steps = min(args.steps, 1000)
         ps.ps_plan_set_timing(pa._plan, n_kernel_steps)
         for _ in range(n_kernel_steps):
@@ -363,6 +475,8 @@ def run_ours(args):
     value = units / (ms * 1e-3) / 1e12
 
     # ---- end to end: host buffers in, host result out, every step ----
+    # Inputs of step i + 1 cross to the device, and the output of step i - 1 crosses back, under the kernels of step
+    # i: two device input buffers and two output buffers, one stream per copy direction, events for the ordering.
     new_k, new_v = [], []
     for r in range(batch.n):
         k, v = gen_cuda.gen_kv(batch.seed, r, int(batch.prior[r]), int(batch.kv_len[r]), s.n_kv_heads, s.head_dim, dev)
@@ -373,6 +487,7 @@ def run_ours(args):
     parts = [db.q.cpu().contiguous().view(torch.uint8).reshape(-1), torch.cat(new_k).cpu().contiguous().view(torch.uint8).reshape(-1),
              torch.cat(new_v).cpu().contiguous().view(torch.uint8).reshape(-1),
              torch.from_numpy(batch.block_table).contiguous().view(torch.uint8).reshape(-1)]
+    del new_k, new_v
     offs, total = [], 0
     for t in parts:
         offs.append(total)
@@ -380,55 +495,94 @@ def run_ours(args):
     h_in = torch.zeros(total, dtype=torch.uint8).pin_memory()
     for t, o in zip(parts, offs):
         h_in[o : o + t.numel()] = t
-    d_in = torch.empty(total, dtype=torch.uint8, device=dev)
+    d_in = [torch.empty(total, dtype=torch.uint8, device=dev) for _ in range(2)]
+    d_out = [torch.empty_like(db.q) for _ in range(2)]
 
-    def view(i, dtype, shape):
-        return d_in[offs[i] : offs[i] + parts[i].numel()].view(dtype).reshape(shape)
+    def view(buf, i, dtype, shape):
+        return buf[offs[i] : offs[i] + parts[i].numel()].view(dtype).reshape(shape)
 
     n_new = int(batch.q_len.sum())
-    d_q = view(0, torch.bfloat16, db.q.shape)
-    d_k = view(1, torch.bfloat16, (n_new, s.n_kv_heads, s.head_dim))
-    d_v = view(2, torch.bfloat16, (n_new, s.n_kv_heads, s.head_dim))
-    d_bt = view(3, torch.int32, db.block_table.shape)
+    views = [(view(b, 0, torch.bfloat16, db.q.shape), view(b, 1, torch.bfloat16, (n_new, s.n_kv_heads, s.head_dim)),
+              view(b, 2, torch.bfloat16, (n_new, s.n_kv_heads, s.head_dim)), view(b, 3, torch.int32, db.block_table.shape))
+             for b in d_in]
     h_out = torch.empty(out.shape, dtype=out.dtype).pin_memory()
     h2d = sum(t.numel() for t in parts)
     d2h = h_out.numel() * 2
+    s_in, s_out = torch.cuda.Stream(dev), torch.cuda.Stream(dev)
 
-    def e2e_step():
-        d_in.copy_(h_in, non_blocking=True)
-        pa.write(d_k, d_v, d_bt, batch.prior, batch.q_len, max_pages=batch.max_pages)
-        pa.plan(batch.prior, batch.q_len, batch.max_pages)
-        pa.run(d_q, d_bt, out=out, want_lse=False)
-        h_out.copy_(out, non_blocking=True)
+    def e2e_loop(n):
+        """n steps; returns when the last output copy has been ordered into the compute stream."""
+        ev_in = [torch.cuda.Event() for _ in range(2)]      # inputs of the step using buffer b are on the device
+        ev_read = [torch.cuda.Event() for _ in range(2)]    # the step using buffer b has finished (inputs read, output written)
+        ev_back = [torch.cuda.Event() for _ in range(2)]    # output buffer b has been copied to the host
+        s_in.wait_stream(stream)
 
-    for _ in range(3):
-        e2e_step()
+        def send(i):
+            b = i & 1
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_read[b])
+                d_in[b].copy_(h_in, non_blocking=True)
+                ev_in[b].record(s_in)
+
+        send(0)
+        for i in range(n):
+            b = i & 1
+            if i + 1 < n:
+                send(i + 1)
+            d_q, d_k, d_v, d_bt = views[b]
+            stream.wait_event(ev_in[b])
+            if i >= 2:
+                stream.wait_event(ev_back[b])
+            pa.write(d_k, d_v, d_bt, batch.prior, batch.q_len, max_pages=batch.max_pages)
+            pa.plan(batch.prior, batch.q_len, batch.max_pages)
+            pa.run(d_q, d_bt, out=d_out[b], want_lse=False)
+            ev_read[b].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_read[b])
+                h_out.copy_(d_out[b], non_blocking=True)
+                ev_back[b].record(s_out)
+        stream.wait_event(ev_back[(n - 1) & 1])
+
+    e2e_loop(3)
     barrier()
     ev0.record(stream)
-    for _ in range(args.steps):
-        e2e_step()
+    e2e_loop(args.steps)
     ev1.record(stream)
     barrier()
     e2e_ms, e2e_units = reduce_over_ranks(ev0.elapsed_time(ev1) / args.steps, dec_bytes, world, dev)
     pa.check()
+    pa.plan(batch.prior, batch.q_len, batch.max_pages)
 
     line = None
     if rank == 0:
         peaks = measured_peaks()
-        achieved = dec_bytes / (dec_ms * 1e-3) / 1e9 if dec_ms > 0 else 0.0
-        roof = {"kernel": "decode_kernel", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": achieved / peaks["hbm_gbs"], "traffic": ncu_traffic(args.workload), "peak_source": peaks["source"],
-                "launch_ms": dec_ms, "algorithmic_bytes_per_launch": dec_bytes, "launches_timed": n_timed}
-        pf_tf = pf_flops / (pre_ms * 1e-3) / 1e12 if pf_flops > 0 and pre_ms > 0 else None
-        extra = {"decode_kernel_ms": dec_ms, "prefill_kernel_ms": pre_ms, "merge_kernel_ms": mrg_ms,
-                 "decode_TBps_kernel": achieved / 1e3, "prefill_TFLOPs_kernel": pf_tf,
-                 "prefill_frac_of_bf16_peak": pf_tf / peaks["bf16_tflops"] if pf_tf else None,
-                 "value_frac_of_nominal_8TBps": value / world / 8.0, "host_issue_ms_per_step": host_ms,
-                 "decode_sms": info.decode_sms, "prefill_sms": info.prefill_sms,
-                 "side_by_side": bool(pf_flops > 0 and dec_bytes > 0 and info.decode_sms + info.prefill_sms <= 148
-                                      and info.decode_sms != info.prefill_sms)}
-        if pf_flops > 0 and dec_bytes > 0:
-            extra.update(components_alone(pa, batch, db, out, args.steps, peaks))
+        # the step against the resource that bounds it when its two kernels overlap perfectly
+        t_hbm = dec_bytes / (peaks["hbm_gbs"] * 1e9)
+        t_tensor = pf_flops / (peaks["bf16_tflops"] * 1e12)
+        mixed = pf_flops > 0 and dec_bytes > 0
+        side_by_side = bool(mixed and info.decode_sms != info.prefill_sms)
+        where = "mixed step, beside the other kernel" if side_by_side else "whole step"
+        kernels = []
+        if dec_bytes > 0:
+            kernels.append(kernel_record("decode_kernel", where + " (%d SMs)" % info.decode_sms, dec_ms, dec_bytes, peaks))
+        if pf_flops > 0:
+            kernels.append(kernel_record("prefill_kernel", where + " (%d SMs)" % info.prefill_sms, pre_ms, pf_flops, peaks))
+        if mixed:
+            kernels.extend(components_alone(pa, batch, db, out, args.steps, peaks))
+        if t_hbm >= t_tensor:
+            ach = dec_bytes / (ms * 1e-3) / 1e9
+            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                    "traffic": ncu_traffic("decode_kernel", dec_bytes), "dominant_kernel": "decode_kernel"}
+        else:
+            ach = pf_flops / (ms * 1e-3) / 1e12
+            roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": ach / peaks["bf16_tflops"], "traffic": ncu_traffic("prefill_kernel", pf_flops),
+                    "dominant_kernel": "prefill_kernel"}
+        roof.update({"peak_source": peaks["source"], "of": "the whole step (ms_per_step)",
+                     "bound_times_ms": {"hbm": t_hbm * 1e3, "tensor": t_tensor * 1e3},
+                     "traffic_source": NCU_TRAFFIC_SOURCE, "launches_timed": n_timed, "merge_kernel_ms": mrg_ms,
+                     "kernels": kernels})
         line = {
             "metric": METRIC, "value": value, "unit": "TB/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "strong" if args.shard == "heads" and world > 1 else "weak",
@@ -436,24 +590,26 @@ def run_ours(args):
             "config": {"workload": desc, "kv_bytes_per_step_per_gpu": dec_bytes, "prefill_flops_per_step_per_gpu": pf_flops,
                        "l2": "inputs larger than L2 (%.0f MB of KV per step), no flush" % (dec_bytes / 1e6),
                        "decode_items": info.n_decode_items, "prefill_items": info.n_prefill_items,
-                       "merge_rows": info.n_merge_rows,
+                       "merge_rows": info.n_merge_rows, "decode_sms": info.decode_sms, "prefill_sms": info.prefill_sms,
+                       "side_by_side": side_by_side,
                        "parallelism": ("kv heads x%d" if args.shard == "heads" and world > 1 else "replicas x%d") % world},
+            "prefill_TFLOPs": pf_flops / (ms * 1e-3) / 1e12 if pf_flops > 0 else None,
+            "host_issue_ms_per_step": host_ms,
             "clocks": clocks.summary(),
             "e2e": {"value": e2e_units / (e2e_ms * 1e-3) / 1e12, "unit": "TB/s", "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "note": "per step: new tokens' Q/K/V and block table from pinned host memory, ps_kv_write, plan, run, "
-                            "output back to host; the KV cache of earlier iterations stays in HBM"},
+                            "output back to pinned host memory; the next step's input copy and the previous step's output "
+                            "copy run on their own streams under this step's kernels; the KV cache of earlier iterations "
+                            "stays in HBM"},
             "gpu_launches": args.steps * info.n_launches,
             "roofline": roof,
-            "kernels": extra,
         }
-        # ---- CPU baseline: the oracle as it stands, on the host's cores ----
+        # ---- CPU baseline: the oracle as it stands, on the host's cores, on a bounded sample ----
         if world == 1 and not args.no_cpu_baseline:
-            reqs = oracle_sample(batch)
-            dt, nbytes, threads = time_oracle(batch, reqs)
-            line["cpu_baseline"] = {"value": nbytes / dt / 1e12, "unit": "TB/s", "cores": threads, "kind": "oracle",
-                                    "seconds": dt, "sample": "%d of %d decode requests (%.1f MB of KV), one pass"
-                                    % (len(reqs), batch.n, nbytes / 1e6)}
+            dec, rows = oracle_sample(batch)
+            sample = OracleSample(batch, dec, rows, dev)
+            line["cpu_baseline"] = cpu_baseline_record(batch, sample, sample.time())
         print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
@@ -466,16 +622,16 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=1, choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", type=int, default=4, choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--shard", default="requests", choices=["requests", "heads"],
                     help="what N > 1 ranks split: requests (each rank its own batch; default) or the KV heads of one batch")
     args = ap.parse_args()
     if args.impl == "reference":
-        args.steps = min(args.steps, 5)  # each step is seconds of CPU work
+        args.steps = min(args.steps, 3)  # each step is seconds of CPU work
         return run_reference(args)
     return run_ours(args)
 

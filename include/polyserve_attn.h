@@ -200,8 +200,17 @@ ps_status ps_plan_get_items(const ps_plan *plan, int32_t *decode_items_out, int6
  * a second stream of the plan, beside the prefill kernel on disjoint SMs (the
  * merge kernel then follows the prefill kernel at once, under the decode
  * kernel), and is joined back into `stream` before the call's work is
- * complete in stream order.  Consecutive runs of one plan must be issued to the
- * same stream, or be ordered by the caller: they share the partial buffers.
+ * complete in stream order.
+ * Ordering rule for the workspace: all runs that use one workspace -- of one
+ * plan, re-planned or not, and of different plans that take turns on it --
+ * must be issued to the same stream, or be ordered by the caller.  Under that
+ * rule no host synchronisation is needed between a ps_attn_plan / ps_attn_run
+ * pair and the next, whatever the batches: the two work-list slots sit at
+ * fixed strides that only grow, a run's upload waits for the run two calls
+ * ago that used its slot, and whenever the library cannot rely on that record
+ * (first use of the memory, slots moved because a work list outgrew them,
+ * another plan's run on the workspace in between) the upload is instead
+ * ordered behind everything already on `stream`.
  * The call may be made while `stream` is being captured into a CUDA graph:
  * the upload then becomes a node of the graph on `stream` (each replay copies
  * the plan's staging image again) and the graph replays this plan, with these
@@ -216,9 +225,27 @@ ps_status ps_attn_run(ps_plan *plan, const ps_kv *kv, const void *q_dev, const i
                       void *stream);
 
 /* Synchronises `stream`, then reports what the plan's last run saw on the
- * device: PS_OK, PS_ERR_BOUNDS (a page id outside the pool; that page was
- * skipped) or PS_ERR_TIMEOUT (a bounded wait expired; output is invalid). */
+ * device: PS_OK, PS_ERR_BOUNDS (a page id outside the pool, which was skipped,
+ * or a work record pointing outside the batch, which was not followed; the
+ * output is invalid) or PS_ERR_TIMEOUT (a bounded wait expired; output is
+ * invalid).  The status word lives in the workspace: read it before another
+ * plan runs on the same workspace. */
 ps_status ps_plan_status(ps_plan *plan, void *stream);
+
+/*
+ * Bound, in nanoseconds, of every wait inside this plan's kernels (for a bulk
+ * copy to land, for another warp's hand-over, for a group of MMAs to retire).
+ * A wait that runs out sets the run's status to PS_ERR_TIMEOUT; the warps of
+ * that CTA stop, let the copies and MMAs already in flight finish (bounded
+ * again, by a fixed second), release their tensor memory and return, so the
+ * context stays usable and nothing is left waiting.  Default: 2 s; at most
+ * 4 s (PS_ERR_INVALID beyond, or for a negative value).  Zero makes
+ * a wait give up as soon as it finds its phase incomplete -- in practice the
+ * first wait of every CTA -- which is how the tests reach this path on a
+ * healthy device.  Takes effect at the next ps_attn_run (a captured graph
+ * keeps the value it was captured with).
+ */
+ps_status ps_plan_set_wait_limit(ps_plan *plan, int64_t limit_ns);
 
 /*
  * ps_attn_run without a caller-provided workspace.  (The paper has no
@@ -245,9 +272,12 @@ ps_status ps_plan_status(ps_plan *plan, void *stream);
  * runtime query made with that device current, as it must be at every call);
  * make that first call before starting any stream capture.  All calls on a
  * device share the one array and it keeps whatever the last call left there:
- * each run rewrites the header words that must start at zero, but two runs
- * that overlap on the GPU (different streams, or different plans in flight)
- * would overwrite each other's work list and partials -- serialise them.
+ * each run rewrites the header words that must start at zero.  The array is a
+ * workspace like any other and ps_attn_run's ordering rule applies to it:
+ * issue all calls on a device to one stream (plans may then take turns freely;
+ * the library orders each upload behind the other plan's run), or order them
+ * yourself -- runs that overlap on the GPU would overwrite each other's work
+ * list and partials.  Read ps_plan_status before another plan uses the array.
  */
 #define PS_STATIC_WORKSPACE_BYTES (8u << 20)
 ps_status ps_attn_run_static(ps_plan *plan, const ps_kv *kv, const void *q_dev, const int32_t *block_table_dev,
@@ -285,6 +315,8 @@ typedef struct {
     uint64_t seed_base;           /* draw s of cell c uses seed seed_base + seeds_per_cell * c + s */
     int32_t include_kv_write;     /* != 0: each timed run first appends the batch's new tokens with ps_kv_write
                                      (section 2.1: the pass that computes attention also populates the cache) */
+    double hbm_peak_gbs;          /* denominators of the rows' roofline_frac: memory bandwidth in GB/s and dense bf16 */
+    double bf16_peak_tflops;      /* tensor rate in TFLOP/s, e.g. as measured on the device; 0 = nominal 8000 / 2250 */
 } ps_grid_spec;
 
 typedef struct {
@@ -299,6 +331,11 @@ typedef struct {
     float latency_min_us;
     float latency_max_us;
     float plan_us;            /* host time of ps_attn_plan for this draw */
+    float decode_TBps;        /* decode_bytes / latency: the decode-attention term of section 3.4 as a rate */
+    float prefill_TFLOPs;     /* prefill_flops / latency (both rates are over the whole step, so in a mixed batch
+                                 each is a lower bound on what its kernel reached) */
+    float roofline_frac;      /* max(decode_bytes / hbm peak, prefill_flops / bf16 peak) / latency: 1 means the step
+                                 took what its slower resource needs when the two kernels overlap perfectly */
 } ps_grid_row;
 
 /*

@@ -51,7 +51,8 @@ class ps_grid_spec(ctypes.Structure):
                 ("decode_counts", ctypes.POINTER(ctypes.c_int32)), ("n_decode_counts", ctypes.c_int32),
                 ("mean_ctxs", ctypes.POINTER(ctypes.c_int32)), ("n_mean_ctxs", ctypes.c_int32),
                 ("seeds_per_cell", ctypes.c_int32), ("warmup", ctypes.c_int32), ("iters", ctypes.c_int32),
-                ("seed_base", ctypes.c_uint64), ("include_kv_write", ctypes.c_int32)]
+                ("seed_base", ctypes.c_uint64), ("include_kv_write", ctypes.c_int32),
+                ("hbm_peak_gbs", ctypes.c_double), ("bf16_peak_tflops", ctypes.c_double)]
 
 
 class ps_grid_row(ctypes.Structure):
@@ -59,12 +60,13 @@ class ps_grid_row(ctypes.Structure):
                 ("seed_index", ctypes.c_int32), ("seed", ctypes.c_uint64), ("token_batch", ctypes.c_int32),
                 ("prefill_prior", ctypes.c_int32), ("kv_tokens", ctypes.c_int64), ("decode_bytes", ctypes.c_double),
                 ("prefill_flops", ctypes.c_double), ("latency_us", ctypes.c_float), ("latency_min_us", ctypes.c_float),
-                ("latency_max_us", ctypes.c_float), ("plan_us", ctypes.c_float)]
+                ("latency_max_us", ctypes.c_float), ("plan_us", ctypes.c_float), ("decode_TBps", ctypes.c_float),
+                ("prefill_TFLOPs", ctypes.c_float), ("roofline_frac", ctypes.c_float)]
 
 
 EXPORTS = ["ps_kv_bytes", "ps_kv_alloc", "ps_kv_free", "ps_kv_write", "ps_kv_gather", "ps_kv_status", "ps_attn_plan",
            "ps_plan_free", "ps_plan_get_info", "ps_plan_get_items", "ps_attn_run", "ps_plan_status",
-           "ps_plan_set_timing", "ps_plan_get_timing", "ps_profile_grid", "ps_attn_run_static",
+           "ps_plan_set_timing", "ps_plan_get_timing", "ps_plan_set_wait_limit", "ps_profile_grid", "ps_attn_run_static",
            "ps_last_error", "ps_version"]
 
 _lib = None
@@ -97,6 +99,7 @@ def load() -> ctypes.CDLL:
     lib.ps_plan_status.argtypes = [_vp, _vp]
     lib.ps_attn_run_static.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp]
     lib.ps_plan_set_timing.argtypes = [_vp, _i32]
+    lib.ps_plan_set_wait_limit.argtypes = [_vp, _i64]
     fp = ctypes.POINTER(ctypes.c_float)
     lib.ps_plan_get_timing.argtypes = [_vp, _vp, fp, fp, fp, ctypes.POINTER(_i32)]
     lib.ps_profile_grid.argtypes = [sp, ctypes.POINTER(ps_grid_spec), ctypes.POINTER(ps_grid_row), _i64,
@@ -226,6 +229,10 @@ def ps_plan_status(plan, stream=None):
     _check(load().ps_plan_status(plan, _ptr(stream)))
 
 
+def ps_plan_set_wait_limit(plan, limit_ns: int):
+    _check(load().ps_plan_set_wait_limit(plan, limit_ns))
+
+
 def ps_plan_set_timing(plan, max_runs: int):
     _check(load().ps_plan_set_timing(plan, max_runs))
 
@@ -238,13 +245,13 @@ def ps_plan_get_timing(plan, stream=None):
 
 
 def ps_profile_grid(shape: ps_shape, chunk_sizes, decode_counts, mean_ctxs, seeds_per_cell, warmup, iters, seed_base,
-                    csv_path=None, stream=None, include_kv_write=False):
+                    csv_path=None, stream=None, include_kv_write=False, hbm_peak_gbs=0.0, bf16_peak_tflops=0.0):
     """Returns the list of ps_grid_row in sweep order."""
     ca, cp = _host_i32(chunk_sizes)
     da, dp = _host_i32(decode_counts)
     ma, mp = _host_i32(mean_ctxs)
     spec = ps_grid_spec(cp, ca.shape[0], dp, da.shape[0], mp, ma.shape[0], seeds_per_cell, warmup, iters, seed_base,
-                        int(bool(include_kv_write)))
+                        int(bool(include_kv_write)), float(hbm_peak_gbs), float(bf16_peak_tflops))
     n = ca.shape[0] * da.shape[0] * ma.shape[0] * seeds_per_cell
     rows = (ps_grid_row * n)()
     n_out = _i64(0)

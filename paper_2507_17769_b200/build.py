@@ -47,8 +47,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
 
     def compile_one(src):
         obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
-        extra = os.environ.get("PS_ATTN_NVCC_EXTRA", "").split()  # e.g. -DPS_DECODE_WARPS=6 for tuning sweeps
-        proc = subprocess.run([nvcc] + NVCC_FLAGS + extra + ["-c", src, "-o", obj], capture_output=True, text=True)
+        proc = subprocess.run([nvcc] + NVCC_FLAGS + ["-c", src, "-o", obj], capture_output=True, text=True)
         return src, obj, proc
 
     objs = []

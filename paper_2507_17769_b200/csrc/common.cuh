@@ -97,6 +97,14 @@ constexpr int kPrefillRowsPerItem = 256;
 
 constexpr int kStatusOk = 0, kStatusBounds = 1, kStatusTimeout = 2;
 
+// Device-side waits (on an mbarrier: a bulk copy landing, another warp's hand-over, an MMA group retiring) give up
+// after this long and flag the run instead of holding the GPU; ps_plan_set_wait_limit changes it per plan.
+constexpr int64_t kDefaultWaitLimitNs = 2000000000ll;
+constexpr int64_t kMaxWaitLimitNs = 4000000000ll;  // the kernels time their waits on the low 32 bits of the nanosecond clock
+// After a wait has run out, the copies a warp still has in flight get this long to land before its shared
+// memory is released (independent of the plan's limit, which a test may set to zero).
+constexpr int64_t kDrainLimitNs = 1000000000ll;
+
 struct WsHeader {         // 64 bytes at the start of the workspace
     int32_t status;       // sticky OR of kStatus* seen by any kernel of the run
     int32_t decode_next;  // dynamic work counters
@@ -163,7 +171,8 @@ struct DeviceWork {       // pointers into the workspace for one run
     int32_t* dmerge_cnt;
     float* part_lse;
     float* part_o;
-    int32_t n_units, n_prefill, n_merge;
+    int32_t n_units, n_prefill, n_merge, n_dmerge;
+    int64_t n_part_slots;              // rows of part_lse / part_o
     const int32_t* prefill_cta_start;  // static prefill partition (n_prefill_ctas + 1 entries), unused when 0
     int32_t n_prefill_ctas;
 };
@@ -182,6 +191,8 @@ struct RunArgs {
     int num_sms;
     int dec_sms, pf_sms;  // SMs (= CTAs) for the decode and the prefill kernel
     int32_t total_q;      // q tokens of the batch (rows of q and out)
+    int32_t n_req;        // requests of the batch (rows of the block table)
+    int64_t wait_limit_ns;
 };
 
 ps_status launch_decode(const RunArgs& a);
@@ -221,11 +232,44 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: returns false if the phase did not complete within the limit.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit = 20000000u) {
-    for (uint32_t i = 0; i < limit; ++i)
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint32_t global_timer_lo() {
+    uint32_t t;
+    asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t));
+    return t;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Wait bounded in time: false if the phase did not complete within about limit_ns nanoseconds.  One
+// non-blocking probe first; a limit of zero gives up right after it (the phase must already be complete).
+// Otherwise the suspending form polls, and the clock is read only every kWaitPollsPerClockRead failed polls
+// (it starts at the first such read), so a wait that ends normally never reads it.
+constexpr uint32_t kWaitPollsPerClockRead = 64;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int64_t limit_ns) {
+    if (mbar_test_wait(bar, parity)) return true;
+    if (limit_ns <= 0) return false;
+    uint64_t t0 = 0;
+    for (uint32_t i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-    return false;
+        if (i % kWaitPollsPerClockRead == 0) {
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > (uint64_t)limit_ns) return false;
+        }
+    }
 }
 
 // global -> shared bulk copy; bytes multiple of 16, both addresses 16-byte aligned

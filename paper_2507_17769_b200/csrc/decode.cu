@@ -65,7 +65,17 @@ struct DecodeParams {
     float* part_o;
     int32_t Hq, Hkv, G;
     float scale_log2;  // log2(e) / sqrt(d)
+    int32_t n_req, total_q, n_dmerge;  // extents the work records are checked against
+    int64_t n_part_slots;
+    int64_t wait_limit_ns;
 };
+
+// A work record that points outside the batch (it can only come from a damaged work list) is replaced by one that
+// stays inside it, and the run is flagged: both cursors of a warp apply the same rule to the same record, so they
+// keep agreeing on how many pages it stands for.
+__device__ __forceinline__ bool piece_pages_ok(const int4& a, const DecodeParams& p) {
+    return (uint32_t)a.x < (uint32_t)p.n_req && (uint32_t)a.y < (uint32_t)p.Hkv && a.z >= 0 && a.z < a.w && a.w <= p.max_pages;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodeParams p) {
@@ -116,7 +126,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
                 P_piece = du.piece_begin;
                 P_piece_end = du.piece_end;
             }
-            const int4 a = __ldg(reinterpret_cast<const int4*>(&p.pieces[P_piece]));
+            int4 a = __ldg(reinterpret_cast<const int4*>(&p.pieces[P_piece]));
+            if (!piece_pages_ok(a, p)) a = make_int4(0, 0, 0, 1);  // flagged by the consumer side
             P_page = a.z;
             P_page_end = a.w;
             P_g = a.y;
@@ -339,8 +350,28 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
                 C_piece = du.piece_begin;
                 C_piece_end = du.piece_end;
             }
-            const int4 a = __ldg(reinterpret_cast<const int4*>(&p.pieces[C_piece]));
-            const int4 b = __ldg(reinterpret_cast<const int4*>(&p.pieces[C_piece]) + 1);
+            int4 a = __ldg(reinterpret_cast<const int4*>(&p.pieces[C_piece]));
+            int4 b = __ldg(reinterpret_cast<const int4*>(&p.pieces[C_piece]) + 1);
+            {
+                bool bad = false;
+                if (!piece_pages_ok(a, p)) {
+                    a = make_int4(0, 0, 0, 1);
+                    bad = true;
+                }
+                if ((uint32_t)b.x >= (uint32_t)p.total_q) {
+                    b.x = 0;
+                    bad = true;
+                }
+                if (b.y >= 0 && ((int64_t)b.y + p.G > p.n_part_slots || (uint32_t)b.w >= (uint32_t)p.n_dmerge)) {
+                    b.y = -1;
+                    bad = true;
+                }
+                if (b.z <= (a.w - 1) * kPage) {  // the row's keys end inside the piece's last page or behind it
+                    b.z = a.w * kPage;
+                    bad = true;
+                }
+                if (bad && lane == 0) atomicOr(&p.hdr->status, kStatusBounds);
+            }
             C_g = a.y;
             C_page = a.z;
             C_page_end = a.w;
@@ -364,7 +395,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
         }
 
         const uint32_t stage = n_cons % STAGES;
-        if (!mbar_wait(bar0 + 8 * stage, (n_cons / STAGES) & 1)) {
+        if (!mbar_wait(bar0 + 8 * stage, (n_cons / STAGES) & 1, p.wait_limit_ns)) {
             if (lane == 0) atomicOr(&p.hdr->status, kStatusTimeout);
             timed_out = true;
             break;
@@ -445,8 +476,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
         for (int k = 0; k < n_deferred; ++k) combine(deferred[3 * k], deferred[3 * k + 1], deferred[3 * k + 2]);
     }
     if (timed_out) {
-        // let copies still in flight land before the CTA's shared memory is released
-        for (uint32_t n = n_cons + 1; n < n_prod; ++n) mbar_wait(bar0 + 8 * (n % STAGES), (n / STAGES) & 1, 2000000u);
+        // let the copies still in flight (the one waited for included) land before the CTA's shared memory is released
+        for (uint32_t n = n_cons; n < n_prod; ++n) mbar_wait(bar0 + 8 * (n % STAGES), (n / STAGES) & 1, kDrainLimitNs);
     }
 }
 
@@ -483,6 +514,11 @@ static ps_status launch_decode_d(const RunArgs& a) {
     p.Hkv = a.shape.n_kv_heads;
     p.G = p.Hq / p.Hkv;
     p.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+    p.n_req = a.n_req;
+    p.total_q = a.total_q;
+    p.n_dmerge = a.w.n_dmerge;
+    p.n_part_slots = a.w.n_part_slots;
+    p.wait_limit_ns = a.wait_limit_ns;
     int grid = (a.w.n_units + kWarps - 1) / kWarps;
     if (grid > a.dec_sms) grid = a.dec_sms;
     decode_kernel<D><<<grid, kWarps * 32, Cfg::kSmemBytes, a.stream>>>(p);

@@ -8,7 +8,11 @@
 #include <cmath>
 #include <cstring>
 #include <functional>
+#include <iterator>
+#include <atomic>
+#include <mutex>
 #include <new>
+#include <unordered_map>
 #include <utility>
 #include <vector>
 
@@ -65,6 +69,43 @@ static inline bool runs_as_decode(const ps_shape& sh, bool tiny_as_rows, int pri
 
 using namespace ps;
 
+namespace {
+
+// Which plan last put a work list into a given workspace.  Two plans that take turns on one workspace (or on the
+// built-in scratch of ps_attn_run_static) each keep their own record of the slots they have used; a plan that finds
+// another plan's serial here orders its upload behind everything already on the caller's stream instead of trusting
+// that record.
+std::mutex g_ws_mu;
+std::unordered_map<const void*, uint64_t> g_ws_owner;
+constexpr size_t kWsOwnerCap = 4096;  // forgetting an entry only costs its next run one stream fence
+
+uint64_t next_plan_serial() {
+    static std::atomic<uint64_t> next{1};
+    return next.fetch_add(1, std::memory_order_relaxed);
+}
+
+// true if `serial` was already the last user of `ws`; records it as the last user either way
+bool claim_workspace(const void* ws, uint64_t serial) {
+    std::lock_guard<std::mutex> lock(g_ws_mu);
+    auto it = g_ws_owner.find(ws);
+    if (it != g_ws_owner.end()) {
+        const bool same = it->second == serial;
+        it->second = serial;
+        return same;
+    }
+    if (g_ws_owner.size() >= kWsOwnerCap) g_ws_owner.clear();
+    g_ws_owner.emplace(ws, serial);
+    return false;
+}
+
+void forget_plan(uint64_t serial) {
+    std::lock_guard<std::mutex> lock(g_ws_mu);
+    for (auto it = g_ws_owner.begin(); it != g_ws_owner.end();)
+        it = it->second == serial ? g_ws_owner.erase(it) : std::next(it);
+}
+
+}  // namespace
+
 struct ps_plan {
     ps_shape shape{};
     int32_t n = 0, max_pages = 0, num_sms = 0, device_sms = 0;
@@ -83,9 +124,15 @@ struct ps_plan {
     std::vector<int32_t> prefill_cta_start;  // static partition: CTA b runs items [start[b], start[b+1]); empty = dynamic queue
     std::vector<int32_t> prior;  // kept for item inspection
     ps_plan_info info{};
-    // workspace layout
+    // workspace layout: two image slots of slot_stride bytes each, then the partial rows.  The stride only ever
+    // grows (with headroom), so that re-planning to another batch normally leaves the slots and the partial
+    // buffers where the runs still in flight expect them.
     size_t off_pieces = 0, off_units = 0, off_prefill = 0, off_merge = 0, off_cta_start = 0, off_dmerge = 0, off_dmerge_cnt = 0, image_bytes = 0;
+    size_t slot_stride = 0;
     size_t off_part_lse = 0, off_part_o = 0, ws_bytes = 0;
+    bool layout_moved = false;  // slot_stride grew since the last run: the slots of earlier runs lie elsewhere
+    uint64_t serial = 0;        // identifies this plan object among all that may share a workspace
+    int64_t wait_limit_ns = kDefaultWaitLimitNs;  // bound of every device-side wait of this plan's kernels
     // pinned staging image of [0, image_bytes)
     char* pinned = nullptr;
     bool pinned_is_cuda = false;
@@ -428,6 +475,7 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     if (fresh) {
         pl = new (std::nothrow) ps_plan();
         if (!pl) return fail(PS_ERR_OOM, "host allocation failed");
+        pl->serial = next_plan_serial();
     } else if (pl->copy_pending && pl->ev_copied[pl->last_slot]) {
         cudaError_t e = cudaEventSynchronize(pl->ev_copied[pl->last_slot]);
         if (e != cudaSuccess) return fail(PS_ERR_CUDA, "cudaEventSynchronize failed: %s", cudaGetErrorString(e));
@@ -532,7 +580,13 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
     pl->off_dmerge_cnt = off; off = align_up(off + pl->dmerge.size() * sizeof(int32_t), 256);
     pl->off_cta_start = off; off = align_up(off + pl->prefill_cta_start.size() * sizeof(int32_t), 256);
     pl->image_bytes = off;
-    off = 2 * pl->image_bytes;  // two image slots
+    if (pl->image_bytes > pl->slot_stride) {
+        // (re)size the slots with headroom: a batch of the next iterations that needs a somewhat longer work list
+        // still fits, and the layout stays put
+        pl->slot_stride = align_up(pl->image_bytes + pl->image_bytes / 2, 4096);
+        pl->layout_moved = true;
+    }
+    off = 2 * pl->slot_stride;  // two image slots
     pl->off_part_lse = off; off = align_up(off + (size_t)n_slots * sizeof(float), 256);
     pl->off_part_o = off;   off = align_up(off + (size_t)n_slots * d * sizeof(float), 256);
     pl->ws_bytes = off;
@@ -601,6 +655,7 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
 
 ps_status ps_plan_free(ps_plan* pl) {
     if (!pl) return PS_OK;
+    forget_plan(pl->serial);
     if (pl->copy_stream) {
         cudaStreamSynchronize(pl->copy_stream);
         cudaStreamDestroy(pl->copy_stream);
@@ -665,40 +720,51 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     if (memcmp(&pool.shape, &pl->shape, sizeof(ps_shape)) != 0) return fail(PS_ERR_INVALID, "plan and pool shapes differ");
     cudaStream_t s = (cudaStream_t)stream;
     char* const ws_base = (char*)workspace_dev;
-    const int slot = (int)(pl->run_no++ & 1u);
-    char* ws = ws_base + (size_t)slot * pl->image_bytes;  // this run's image slot; partials are addressed from ws_base
+    const int slot = (int)(pl->run_no & 1u);
+    char* ws = ws_base + (size_t)slot * pl->slot_stride;  // this run's image slot; partials are addressed from ws_base
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     PS_CUDA_TRY(cudaStreamIsCapturing(s, &cap));
     const bool capturing = cap != cudaStreamCaptureStatusNone;
+    // The upload may run under the kernels of the previous run only if this plan's own record of the two slots is
+    // all there is to know about the workspace: same memory as last time, slots where they were, and no other
+    // plan's run on it since.
+    const bool mine = claim_workspace(workspace_dev, pl->serial);
+    const bool known = mine && pl->last_ws == workspace_dev && !pl->layout_moved;
     if (capturing) {
         // Inside a stream capture the upload is a node of the graph on the caller's stream: every replay copies the
         // staging image as it then stands.  Nothing recorded here may be waited for by a later call outside the
         // capture, so the slot bookkeeping starts afresh.
         PS_CUDA_TRY(cudaMemcpyAsync(ws, pl->pinned, pl->image_bytes, cudaMemcpyHostToDevice, s));
         pl->done_valid[0] = pl->done_valid[1] = false;
-        pl->last_ws = workspace_dev;
     } else if (pl->copy_stream) {
         cudaStream_t cs = pl->copy_stream;
-        if (pl->last_ws == workspace_dev && pl->done_valid[slot]) {
-            // same workspace as before: the slot is free once the run two calls ago has finished
+        if (known && pl->done_valid[slot]) {
+            // the slot is free once the run two calls ago has finished; the previous run reads the other slot and
+            // the partial rows behind both
             PS_CUDA_TRY(cudaStreamWaitEvent(cs, pl->ev_done[slot], 0));
         } else {
-            // first use of this memory: order the upload after everything already on the caller's stream
+            // First use of this memory, slots that have moved, or another plan's work list in it: the upload is
+            // ordered after everything already on the caller's stream (every earlier run that shares this workspace
+            // is on that stream, or ordered before this call by the caller).
             PS_CUDA_TRY(cudaEventRecord(pl->ev_fence, s));
             PS_CUDA_TRY(cudaStreamWaitEvent(cs, pl->ev_fence, 0));
-            if (pl->last_ws != workspace_dev) pl->done_valid[0] = pl->done_valid[1] = false;
+            if (!known) pl->done_valid[0] = pl->done_valid[1] = false;
         }
         PS_CUDA_TRY(cudaMemcpyAsync(ws, pl->pinned, pl->image_bytes, cudaMemcpyHostToDevice, cs));
         PS_CUDA_TRY(cudaEventRecord(pl->ev_copied[slot], cs));
         PS_CUDA_TRY(cudaStreamWaitEvent(s, pl->ev_copied[slot], 0));
         pl->copy_pending = true;
         pl->last_slot = slot;
-        pl->last_ws = workspace_dev;
     } else {
         PS_CUDA_TRY(cudaMemcpyAsync(ws, pl->pinned, pl->image_bytes, cudaMemcpyHostToDevice, s));
         PS_CUDA_TRY(cudaStreamSynchronize(s));  // no event to guard the staging image: finish the copy now
     }
+    // the upload is in place (or queued): only now does the run count
+    ++pl->run_no;
+    pl->layout_moved = false;
+    pl->last_ws = workspace_dev;
     pl->last_hdr = (WsHeader*)ws;
+    pl->done_valid[slot] = false;  // until this run's own completion event is recorded below
 
     RunArgs a{};
     a.shape = pl->shape;
@@ -713,7 +779,9 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     a.num_sms = pl->num_sms;
     a.dec_sms = pl->dec_sms;
     a.pf_sms = pl->pf_sms;
-    a.total_q = pl->info.total_q_tokens;
+    a.total_q = (int32_t)pl->info.total_q_tokens;
+    a.n_req = pl->n;
+    a.wait_limit_ns = pl->wait_limit_ns;
     a.w.hdr = (WsHeader*)ws;
     a.w.pieces = (const DecodePiece*)(ws + pl->off_pieces);
     a.w.units = (const DecodeUnit*)(ws + pl->off_units);
@@ -724,6 +792,8 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
     a.w.n_units = (int32_t)pl->units.size();
     a.w.n_prefill = (int32_t)pl->prefill.size();
     a.w.n_merge = (int32_t)pl->merge.size();
+    a.w.n_dmerge = (int32_t)pl->dmerge.size();
+    a.w.n_part_slots = pl->info.n_partial_slots;
     a.w.dmerge = (const DecodeMerge*)(ws + pl->off_dmerge);
     a.w.dmerge_cnt = (int32_t*)(ws + pl->off_dmerge_cnt);
     a.w.prefill_cta_start = (const int32_t*)(ws + pl->off_cta_start);
@@ -741,36 +811,37 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
         cudaStream_t side = pl->side_stream;
         PS_CUDA_TRY(cudaEventRecord(pl->ev_fork, s));
         PS_CUDA_TRY(cudaStreamWaitEvent(side, pl->ev_fork, 0));
+        // From here on the side stream belongs to this call (inside a capture: to the capture): whatever
+        // fails below, it is joined back into the caller's stream before the call returns.
         if (rec) cudaEventRecord(ev[2], side);
         RunArgs ad = a;
         ad.stream = side;
         st = launch_decode(ad);
-        if (st != PS_OK) return st;
-        if (rec) cudaEventRecord(ev[3], side);
-        if (rec) cudaEventRecord(ev[0], s);
-        st = launch_prefill(a);
-        if (st != PS_OK) return st;
-        if (rec) cudaEventRecord(ev[1], s);
-        if (!(a.w.n_prefill_ctas == 0 && a.w.n_prefill > a.pf_sms)) {
+        if (rec && st == PS_OK) cudaEventRecord(ev[3], side);
+        if (rec && st == PS_OK) cudaEventRecord(ev[0], s);
+        if (st == PS_OK) st = launch_prefill(a);
+        if (rec && st == PS_OK) cudaEventRecord(ev[1], s);
+        const bool helpers = a.w.n_prefill_ctas == 0 && a.w.n_prefill > a.pf_sms;
+        if (st == PS_OK && !helpers) {
             // Only this launch writes prefill partials: combine them right behind it, on the SMs it leaves, while
             // the decode kernel is still streaming (decode rows are combined inside the decode kernel).
             if (rec) cudaEventRecord(ev[4], s);
             st = launch_merge(a);
-            if (st != PS_OK) return st;
             if (rec) cudaEventRecord(ev[5], s);
             merged = true;
         }
-        if (a.w.n_prefill_ctas == 0 && a.w.n_prefill > a.pf_sms) {
+        if (st == PS_OK && helpers) {
             // dynamic item queue: once the decode CTAs have left their SMs, as many more prefill CTAs
             // start there and help drain the same queue
             RunArgs ah = a;
             ah.stream = side;
             ah.pf_sms = a.dec_sms;
             st = launch_prefill(ah);
-            if (st != PS_OK) return st;
         }
-        PS_CUDA_TRY(cudaEventRecord(pl->ev_join, side));
-        PS_CUDA_TRY(cudaStreamWaitEvent(s, pl->ev_join, 0));
+        const cudaError_t ej = cudaEventRecord(pl->ev_join, side);
+        const cudaError_t ew = ej == cudaSuccess ? cudaStreamWaitEvent(s, pl->ev_join, 0) : ej;
+        if (st != PS_OK) return st;
+        PS_CUDA_TRY(ew);
     } else {
         if (rec) cudaEventRecord(ev[0], s);
         st = launch_prefill(a);
@@ -792,6 +863,14 @@ ps_status ps_attn_run(ps_plan* pl, const ps_kv* kv, const void* q_dev, const int
         pl->done_valid[slot] = true;
     }
     return st;
+}
+
+ps_status ps_plan_set_wait_limit(ps_plan* pl, int64_t limit_ns) {
+    if (!pl) return fail(PS_ERR_INVALID, "null argument");
+    if (limit_ns < 0 || limit_ns > kMaxWaitLimitNs)
+        return fail(PS_ERR_INVALID, "limit_ns=%lld outside [0, %lld]", (long long)limit_ns, (long long)kMaxWaitLimitNs);
+    pl->wait_limit_ns = limit_ns;
+    return PS_OK;
 }
 
 ps_status ps_plan_set_timing(ps_plan* pl, int32_t max_runs) {

@@ -183,22 +183,25 @@ struct PrefillCfg {
     static constexpr uint32_t kColS = 0, kColO = 256, kColTile = 128;  // tile X at + X * 128
 };
 
+// Kept within 128 bytes: a larger parameter block makes the compiler copy it (and the tensor map) to the stack.
 struct PrefillParams {
     const char* pool;
-    int64_t num_pages;
     const int32_t* block_table;
-    int32_t max_pages;
     __nv_bfloat16* out;
     float* lse;
     WsHeader* hdr;
     const PrefillItem* items;
-    int32_t n_items;
     const int32_t* cta_start;  // static partition: this CTA runs items [cta_start[b], cta_start[b + 1]); null = dynamic queue
     float* part_lse;
     float* part_o;
+    int64_t num_pages;
+    uint32_t wait_limit_ns;
+    int32_t max_pages;
+    int32_t n_items;
     int32_t Hq, Hkv, G;
-    float scale_log2;
+    int32_t n_req, total_q, n_part_slots;  // extents the item records are checked against
 };
+static_assert(sizeof(PrefillParams) <= 128, "parameter block");
 
 constexpr int kItemRing = 4;        // item records in flight between the producer and the other roles
 constexpr int kConsumerWarps = 9;   // eight softmax warps and the MMA warp read every record
@@ -207,24 +210,38 @@ struct Bars {  // byte offsets from the barrier block; [2] = one per stage or pe
     static constexpr int k_full = 0, k_empty = 16, v_full = 32, v_empty = 48, s_full = 64, p_ready = 80, o_done = 96;
     static constexpr int q_full = 112, q_empty = 128, item_full = 144, item_empty = item_full + 8 * kItemRing;
     static constexpr int tmem_slot = item_empty + 8 * kItemRing, abort_slot = tmem_slot + 4;
+    static constexpr int limit_slot = abort_slot + 4;   // wait limit in ns, directly behind the abort flag
+    static constexpr int mma_drained = limit_slot + 8;  // after an abort: the MMAs issued so far have retired
+    static constexpr int armed = mma_drained + 8;       // 6 ints: parity of the last phase armed with copies (K, V stages, Q tiles)
     static constexpr int ring = 256;  // kItemRing PrefillItem records
     static constexpr int bytes = ring + kItemRing * (int)sizeof(PrefillItem);
 };
-static_assert(Bars::abort_slot + 4 <= Bars::ring && sizeof(PrefillItem) == 32 && Bars::bytes <= kBarBlockBytes, "barrier block layout");
+static_assert(Bars::mma_drained % 8 == 0 && Bars::armed + 24 <= Bars::ring && sizeof(PrefillItem) == 32 &&
+                  Bars::bytes <= kBarBlockBytes,
+              "barrier block layout");
 
+// Wait for a phase for at most about the CTA's wait limit (nanoseconds, in the word behind the abort flag; the low
+// half of the nanosecond clock serves, so limits reach 4 s); gives up early when another role of the CTA has already
+// given up.  The role whose wait runs out raises the CTA's abort flag.  One non-blocking probe first; a limit of
+// zero gives up right after it.  The clock is read only every kWaitPollsPerClockRead failed polls.
 __device__ __forceinline__ bool wait_or_abort(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t i = 0; i < 40000000u; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 1023u) == 1023u && *abort_flag) return false;
+    if (mbar_test_wait(bar, parity)) return true;
+    const uint32_t limit_ns = (uint32_t)abort_flag[1];  // the wait limit sits behind the abort flag
+    if (limit_ns > 0) {
+        uint32_t t0 = 0;
+        for (uint32_t i = 1;; ++i) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if ((i & (kWaitPollsPerClockRead - 1)) == 0) {
+                if (*abort_flag) return false;
+                const uint32_t now = global_timer_lo() | 1u;
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > limit_ns) break;
+            }
+        }
     }
     *abort_flag = 1;
     return false;
 }
-// warp-uniform result, so that the warp-collective instructions that follow stay converged
-__device__ __forceinline__ bool wait_all(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    return __all_sync(0xffffffffu, wait_or_abort(bar, parity, abort_flag));
-}
-
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap q_map) {
     using Cfg = PrefillCfg<D>;
@@ -235,6 +252,9 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
     volatile int* s_tmem = reinterpret_cast<volatile int*>(smem + Cfg::kOffBar + Bars::tmem_slot);
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + Cfg::kOffBar + Bars::abort_slot);
     uint4* ring = reinterpret_cast<uint4*>(smem + Cfg::kOffBar + Bars::ring);  // two uint4 per record
+    // written by the producer's lane 0: parity of the last phase of each K / V stage and Q buffer that it armed with
+    // copies (-1: none yet); read only after an abort
+    volatile int* const s_armed = reinterpret_cast<volatile int*>(smem + Cfg::kOffBar + Bars::armed);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
@@ -253,8 +273,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
             mbar_init(bars + Bars::item_full + 8 * s, 1);
             mbar_init(bars + Bars::item_empty + 8 * s, kConsumerWarps);
         }
+        mbar_init(bars + Bars::mma_drained, 1);
         mbar_fence_init();
         *s_abort = 0;
+        s_abort[1] = (int)p.wait_limit_ns;
+        for (int k = 0; k < 6; ++k) s_armed[k] = -1;
     }
     if (warp == 0) {
         tmem_alloc(bars + Bars::tmem_slot, Cfg::kTmemCols);
@@ -264,6 +287,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = (uint32_t)*s_tmem;
+    // warp-uniform result, so that the warp-collective instructions that follow stay converged
+    auto wait_all = [](uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+        return __all_sync(0xffffffffu, wait_or_abort(bar, parity, abort_flag));
+    };
 
     // The roles never meet at a CTA-wide barrier after this point: items flow through the record ring
     // and the mbarriers, so the next item's Q, K and first QK^T overlap the current item's last
@@ -274,6 +301,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
     static_assert(kPrefillRowsPerItem == 2 * kRows, "the planner pairs two q tiles per item");
     const int tile_tok = kRows / p.G;
     const int g_shift = 31 - __clz(p.G);  // G is a power of two
+    constexpr float kScaleLog2 = D == 128 ? 0.12751743f : 0.18033688f;  // log2(e) / sqrt(D)
 
     // consumer side of the record ring: record number n into `it`; false at the end-of-work record or on abort
     auto take_item = [&](uint32_t n, PrefillItem& it) -> bool {
@@ -352,7 +380,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                                 mx3 = max3(mx3, __uint_as_float(sv[q][c + 6]), __uint_as_float(sv[q][c + 7]));
                             }
                     }
-                    const float mx_s = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+                    const float mx_s = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * kScaleLog2;
                     float m_new = m;
                     if (mx_s > m + kRescaleThreshold) m_new = mx_s;  // also the first finite max (m = -inf)
                     const float alpha = (m_new == m) ? 1.f : fast_exp2(m - m_new);
@@ -388,8 +416,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                                 const int q = hhalf * 2 + qq;
 #pragma unroll
                                 for (int c = 0; c < 32; c += 2) {
-                                    float p0 = fast_exp2(fmaf(__uint_as_float(sv[q][c]), p.scale_log2, -m_sub));
-                                    float p1 = fast_exp2(fmaf(__uint_as_float(sv[q][c + 1]), p.scale_log2, -m_sub));
+                                    float p0 = fast_exp2(fmaf(__uint_as_float(sv[q][c]), kScaleLog2, -m_sub));
+                                    float p1 = fast_exp2(fmaf(__uint_as_float(sv[q][c + 1]), kScaleLog2, -m_sub));
                                     p0 = (q * 32 + c < vis) ? p0 : 0.f;
                                     p1 = (q * 32 + c + 1 < vis) ? p1 : 0.f;
                                     const uint32_t pk = pack_bf16(p0, p1);
@@ -402,7 +430,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                         }
                     } else {
                         // Interior tiles: two scores per instruction (packed fp32 FMA and add); four sum chains.
-                        const uint64_t sc2 = pack2(p.scale_log2, p.scale_log2), nm2 = pack2(-m_sub, -m_sub);
+                        const uint64_t sc2 = pack2(kScaleLog2, kScaleLog2), nm2 = pack2(-m_sub, -m_sub);
                         uint64_t ls0 = 0ull, ls1 = 0ull;
 #pragma unroll
                         for (int hhalf = 0; hhalf < 2; ++hhalf) {
@@ -557,6 +585,19 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                     const uint4* src = reinterpret_cast<const uint4*>(p.items + idx);
                     rec0 = __ldg(src);
                     rec1 = __ldg(src + 1);
+                    // A record that points outside the batch (only a damaged work list has one) ends this CTA's
+                    // work and flags the run; nothing is read or written through it.
+                    const int32_t r_req = (int32_t)rec0.x, r_g = (int32_t)rec0.y, r_kb = (int32_t)rec0.z, r_ke = (int32_t)rec0.w;
+                    const int32_t r_q = (int32_t)rec1.x, r_n = (int32_t)rec1.y, r_slot = (int32_t)rec1.z, r_pos = (int32_t)rec1.w;
+                    const bool rec_ok = (uint32_t)r_req < (uint32_t)p.n_req && (uint32_t)r_g < (uint32_t)p.Hkv && r_kb >= 0 &&
+                                        r_kb % kTileKeys == 0 && r_kb < r_ke && r_ke <= p.max_pages * kPage && r_n >= 1 &&
+                                        r_n <= 2 * tile_tok && r_q >= 0 && (int64_t)r_q + r_n <= p.total_q && r_pos >= 0 &&
+                                        (int64_t)r_pos + r_n >= r_ke &&
+                                        (r_slot < 0 || (int64_t)r_slot + (int64_t)r_n * p.G <= p.n_part_slots);
+                    if (!rec_ok) {
+                        if (lane == 0) atomicOr(&p.hdr->status, kStatusBounds);
+                        rec0 = rec1 = make_uint4(0, 0, 0, 0);
+                    }
                 }
                 const uint32_t slot = n_item % kItemRing;
                 ok = wait_all(bars + Bars::item_empty + 8 * slot, ((n_item / kItemRing) & 1) ^ 1, s_abort);
@@ -590,7 +631,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
 
                     ok = wait_all(bars + Bars::k_empty + 8 * s, par ^ 1, s_abort);
                     if (!ok) break;
-                    if (lane == 0) mbar_expect_tx(bars + Bars::k_full + 8 * s, tile_bytes);
+                    if (lane == 0) {
+                        mbar_expect_tx(bars + Bars::k_full + 8 * s, tile_bytes);
+                        s_armed[s] = (int)par;
+                    }
                     __syncwarp();
                     if (mine && which < Cfg::kHalves)
                         bulk_g2s_hint(sbase + Cfg::kOffK + s * Cfg::kKBytes + which * Cfg::kHalfBytes + pg * kPieceBytes,
@@ -606,6 +650,7 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                             if (!ok) break;
                             if (lane == 0) {
                                 mbar_expect_tx(bars + Bars::q_full + 8 * x, Cfg::kQBytes);
+                                s_armed[4 + x] = (int)(items_x[x] & 1);
 #pragma unroll
                                 for (int h = 0; h < Cfg::kHalves; ++h)
                                     tma_load_3d(sbase + Cfg::kOffQ + x * Cfg::kQBytes + h * Cfg::kHalfBytes, &q_map, h * 64,
@@ -618,7 +663,10 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
 
                     ok = wait_all(bars + Bars::v_empty + 8 * s, par ^ 1, s_abort);
                     if (!ok) break;
-                    if (lane == 0) mbar_expect_tx(bars + Bars::v_full + 8 * s, tile_bytes);
+                    if (lane == 0) {
+                        mbar_expect_tx(bars + Bars::v_full + 8 * s, tile_bytes);
+                        s_armed[2 + s] = (int)par;
+                    }
                     __syncwarp();
                     if (mine && which >= 2 && which - 2 < Cfg::kHalves)
                         bulk_g2s_hint(sbase + Cfg::kOffV + s * Cfg::kVBytes + (which - 2) * Cfg::kHalfBytes + pg * kPieceBytes,
@@ -734,17 +782,29 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
         // (the warpgroup's two other warps have no work; they wait at the final barrier)
     }
 
-    // after an abort: flag the run and give copies in flight a bounded time to land
-    if (*s_abort) {
-        if (threadIdx.x == 0) atomicOr(&p.hdr->status, kStatusTimeout);
-        for (int s = 0; s < 2; ++s) {
-            mbar_wait(bars + Bars::k_full + 8 * s, 0, 200000u);
-            mbar_wait(bars + Bars::v_full + 8 * s, 0, 200000u);
-            mbar_wait(bars + Bars::q_full + 8 * s, 0, 200000u);
-        }
-    }
     tc_fence_before();
-    __syncthreads();
+    __syncthreads();  // every role has left its loop
+    if (*s_abort) {
+        // A bounded wait ran out somewhere in this CTA: the output is invalid and the run is flagged.  Before the CTA
+        // gives back its shared and tensor memory, the copies the producer has requested get a bounded time to land
+        // and the MMAs issued so far (they read shared memory and write tensor memory) to retire.
+        if (threadIdx.x == 0) atomicOr(&p.hdr->status, kStatusTimeout);
+        if (warp == kProducerWarp) {
+            for (int k = 0; k < 2; ++k) {
+                const int ak = s_armed[k], av = s_armed[2 + k], aq = s_armed[4 + k];
+                if (ak >= 0) mbar_wait(bars + Bars::k_full + 8 * k, (uint32_t)ak, kDrainLimitNs);
+                if (av >= 0) mbar_wait(bars + Bars::v_full + 8 * k, (uint32_t)av, kDrainLimitNs);
+                if (aq >= 0) mbar_wait(bars + Bars::q_full + 8 * k, (uint32_t)aq, kDrainLimitNs);
+            }
+        }
+        if (warp == kMmaWarp) {
+            if (elect_one()) tc_commit(bars + Bars::mma_drained);
+            __syncwarp();
+            mbar_wait(bars + Bars::mma_drained, 0, kDrainLimitNs);
+        }
+        tc_fence_before();
+        __syncthreads();
+    }
     if (warp == 0) tmem_dealloc(tmem, Cfg::kTmemCols);
 }
 
@@ -796,7 +856,10 @@ static ps_status launch_prefill_d(const RunArgs& a) {
     p.Hq = a.shape.n_q_heads;
     p.Hkv = a.shape.n_kv_heads;
     p.G = p.Hq / p.Hkv;
-    p.scale_log2 = 1.4426950408889634f / sqrtf((float)D);
+    p.n_req = a.n_req;
+    p.total_q = a.total_q;
+    p.n_part_slots = (int32_t)a.w.n_part_slots;
+    p.wait_limit_ns = (uint32_t)a.wait_limit_ns;
 
     // Q as a [T tokens][Hq heads][D] tensor; a box is one 64-element half of a q tile's 128 rows
     EncodeTiledFn encode = tensor_map_encoder();

@@ -205,7 +205,7 @@ extern "C" ps_status ps_profile_grid(const ps_shape* shape, const ps_grid_spec* 
             return fail(PS_ERR_INVALID, "cannot open %s for writing", csv_path);
         }
         fprintf(csv, "component,chunk,n_decode,mean_ctx,seed_index,seed,token_batch,prefill_prior,kv_tokens,decode_bytes,"
-                     "prefill_flops,latency_us,latency_min_us,latency_max_us,plan_us\n");
+                     "prefill_flops,latency_us,latency_min_us,latency_max_us,plan_us,decode_TBps,prefill_TFLOPs,roofline_frac\n");
     }
 
     Draw dr;
@@ -282,12 +282,20 @@ extern "C" ps_status ps_profile_grid(const ps_shape* shape, const ps_grid_spec* 
                     r.latency_min_us = times.front();
                     r.latency_max_us = times.back();
                     r.plan_us = (float)std::chrono::duration<double, std::micro>(t1 - t0).count();
+                    {
+                        const double sec = (double)r.latency_us * 1e-6;
+                        const double hbm = (spec->hbm_peak_gbs > 0 ? spec->hbm_peak_gbs : 8000.0) * 1e9;
+                        const double tensor = (spec->bf16_peak_tflops > 0 ? spec->bf16_peak_tflops : 2250.0) * 1e12;
+                        r.decode_TBps = sec > 0 ? (float)(r.decode_bytes / sec / 1e12) : 0.f;
+                        r.prefill_TFLOPs = sec > 0 ? (float)(r.prefill_flops / sec / 1e12) : 0.f;
+                        r.roofline_frac = sec > 0 ? (float)(std::max(r.decode_bytes / hbm, r.prefill_flops / tensor) / sec) : 0.f;
+                    }
                     if (csv)
-                        fprintf(csv, "%s,%d,%d,%d,%d,%llu,%d,%d,%lld,%.0f,%.0f,%.3f,%.3f,%.3f,%.3f\n",
+                        fprintf(csv, "%s,%d,%d,%d,%d,%llu,%d,%d,%lld,%.0f,%.0f,%.3f,%.3f,%.3f,%.3f,%.4f,%.2f,%.4f\n",
                                 spec->include_kv_write ? "attn+kv_write" : "attn", r.chunk, r.n_decode,
                                 r.mean_ctx, r.seed_index, (unsigned long long)r.seed, r.token_batch, r.prefill_prior,
                                 (long long)r.kv_tokens, r.decode_bytes, r.prefill_flops, r.latency_us, r.latency_min_us,
-                                r.latency_max_us, r.plan_us);
+                                r.latency_max_us, r.plan_us, r.decode_TBps, r.prefill_TFLOPs, r.roofline_frac);
                 }
     if (csv) fclose(csv);
     cudaStreamSynchronize(s);

@@ -10,7 +10,7 @@ import paper_2507_17769_b200 as ps
 from paper_2507_17769_b200 import binding as B
 from workloads import gen
 
-from parity_util import compare, oracle_subset
+from parity_util import compare, oracle_in_groups, oracle_subset
 
 pytestmark = pytest.mark.gpu
 
@@ -154,6 +154,8 @@ def test_config1_decode_only_full_parity():
 
 
 def sampled_parity(batch, dec_reqs, chunk_rows, what):
+    """Every output finite; the rows of ``dec_reqs`` (decode requests) and ``chunk_rows`` (request -> new-token
+    indices) against the oracle, which computes them one by one."""
     db = device_batch(batch)
     db.plan()
     out, lse = db.run()
@@ -162,41 +164,49 @@ def sampled_parity(batch, dec_reqs, chunk_rows, what):
 
     assert bool(torch.isfinite(out.float()).all())
     rows = {r: toks for r, toks in chunk_rows.items()}
-    want, want_lse, packed = oracle_subset(batch, list(dec_reqs) + list(chunk_rows.keys()), rows)
+    want, want_lse, packed = oracle_in_groups(batch, list(dec_reqs) + list(chunk_rows.keys()), rows)
     return compare(out, lse, want, want_lse, packed, what=what), db
 
 
-def chunk_sample(c):
-    return sorted(set(list(range(8)) + list(range(c - 8, c)) + list(range(0, c, 64))))
+def chunk_sample(c, edge=8, every=64):
+    return sorted(set(list(range(min(edge, c))) + list(range(max(0, c - edge), c)) + list(range(0, c, every))))
 
 
-def test_config2_mixed_batch_sampled_parity():
+def test_config2_mixed_batch_full_parity():
+    """Every row of config 2 -- all 512 decode rows and all 1536 rows of the chunk -- against the oracle."""
     import torch
 
     b = gen.config2()
-    dec = [0, 1, int(np.argmax(b.kv_len[:512])), int(np.argmin(b.kv_len[:512]))]
-    _, db = sampled_parity(b, dec, {512: chunk_sample(1536)}, "config2")
-    # the two kernels of this batch run side by side on disjoint SMs; the result is still the same bits every run
+    db = device_batch(b)
     info = db.plan()
+    out, lse = db.run()
+    db.pa.check()
+    want, want_lse, packed = oracle_in_groups(b, range(b.n))
+    assert np.array_equal(packed, np.arange(b.total_q))
+    compare(out, lse, want, want_lse, packed, what="config2, all %d rows" % b.total_q)
+    # the two kernels of this batch run side by side on disjoint SMs; the result is still the same bits every run
     assert 0 < info.decode_sms < info.decode_sms + info.prefill_sms and info.decode_sms != info.prefill_sms
-    o1, l1 = db.run()
     o2, l2 = db.run()
     db.pa.check()
-    assert torch.equal(o1, o2) and torch.equal(l1, l2)
+    assert torch.equal(out, o2) and torch.equal(lse, l2)
 
 
-def test_config3_cells_sampled_parity():
-    for chunk, nd, m, seed in [(64, 8, 512, gen.grid_seed(0, 0)), (256, 32, 2048, gen.grid_seed(30, 1)),
-                               (2048, 8, 8192, gen.grid_seed(62, 2))]:
-        b = gen.config3_cell(chunk, nd, m, seed)
-        sampled_parity(b, [0, nd - 1], {nd: chunk_sample(chunk)[:24]}, "config3 cell %d/%d/%d" % (chunk, nd, m))
+def test_config3_every_cell_sampled_parity():
+    """All 72 cells of the latency-table grid at seed index 0: every output finite, and against the oracle all
+    heads of four decode sequences (first, last, longest, shortest) plus the first / last 8 and every 64th row
+    of the chunk."""
+    for cell, chunk, nd, m in gen.grid_cells():
+        b = gen.config3_cell(chunk, nd, m, gen.grid_seed(cell, 0))
+        dec = sorted({0, nd - 1, int(np.argmax(b.kv_len[:nd])), int(np.argmin(b.kv_len[:nd]))})
+        sampled_parity(b, dec, {nd: chunk_sample(chunk)}, "config3 cell %d (%d/%d/%d)" % (cell, chunk, nd, m))
 
 
-def test_config4_large_long_context_sampled_parity():
+def test_config4_large_long_context_dense_parity():
+    """Config 4: every one of the 256 decode rows, and of both 2048-token chunks the first and last 16 rows plus
+    every 16th row, against the oracle; every other output finite."""
     b = gen.config4()
-    dec = [0, int(np.argmax(b.kv_len[:256]))]
-    rows = [0, 1, 2047, 1024]
-    sampled_parity(b, dec, {256: rows, 257: rows[:2]}, "config4")
+    rows = chunk_sample(2048, edge=16, every=16)
+    sampled_parity(b, range(256), {256: rows, 257: rows}, "config4")
 
 
 def test_page_permutation_gives_identical_bits_and_runs_repeat():

@@ -78,3 +78,30 @@ def test_static_scratch_refuses_plans_that_do_not_fit():
         assert "built-in scratch" in str(e.value)
     finally:
         ps.ps_plan_free(plan)
+
+
+def test_static_scratch_two_plans_taking_turns_without_synchronising():
+    """Two plans share the one built-in array on one stream, in the order A, A, B, A, ... with no host
+    synchronisation: a plan's work-list upload must not land on the other plan's run while that is still
+    reading the array."""
+    import torch
+    from workloads.device import DeviceBatch
+
+    a = DeviceBatch(gen.make_batch(gen.SHAPE_8B, 74, [1500, 99, 2100, 10, 333, 800, 1200, 40], [1, 150, 1, 1, 40, 1, 1, 1]))
+    b = DeviceBatch(gen.make_batch(gen.SHAPE_8B, 75, [40, 5, 600], [1, 20, 1]))
+    stream = torch.cuda.current_stream().cuda_stream
+    ref = {}
+    for name, d in (("A", a), ("B", b)):
+        d.plan()
+        ref[name] = d.run()[0]
+        d.pa.check()
+    outs = []
+    for name in "AABABBA" * 10:
+        d = a if name == "A" else b
+        out = torch.empty_like(d.q)
+        B.ps_attn_run_static(d.pa._plan, d.pa.kv, d.q, d.block_table, out, None, stream)
+        outs.append((name, out))
+    torch.cuda.synchronize()
+    a.pa.check()
+    for i, (name, out) in enumerate(outs):
+        assert torch.equal(out.view(torch.int16), ref[name].view(torch.int16)), "call %d (plan %s)" % (i, name)
