@@ -315,6 +315,17 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
         return it.n_tok > 0;
     };
     auto tiles_of = [](const PrefillItem& it) { return (it.key_end - it.key_begin + kTileKeys - 1) / kTileKeys; };
+    // the MMA warp needs only an item's key-tile count and how many q tiles it has (0 q tiles: end of work)
+    auto take_shape = [&](uint32_t n, int& n_tiles, int& n_x) -> bool {
+        const uint32_t slot = n % kItemRing;
+        if (!wait_all(bars + Bars::item_full + 8 * slot, (n / kItemRing) & 1, s_abort)) return false;
+        const uint4 a = ring[2 * slot], b = ring[2 * slot + 1];
+        n_tiles = ((int32_t)a.w - (int32_t)a.z + kTileKeys - 1) / kTileKeys;
+        n_x = (int32_t)b.y > tile_tok ? 2 : 1;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bars + Bars::item_empty + 8 * slot);
+        return (int32_t)b.y > 0;
+    };
 
     if (warp < 8) {
         // ====================================================================
@@ -608,11 +619,11 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                     mbar_arrive(bars + Bars::item_full + 8 * slot);
                 }
                 ++n_item;
-                PrefillItem it;
+                struct { int32_t req, kv_head, key_begin, key_end, q_tok, n_tok; } it;
                 it.req = (int32_t)rec0.x, it.kv_head = (int32_t)rec0.y, it.key_begin = (int32_t)rec0.z, it.key_end = (int32_t)rec0.w;
-                it.q_tok = (int32_t)rec1.x, it.n_tok = (int32_t)rec1.y, it.part_slot = (int32_t)rec1.z, it.first_pos = (int32_t)rec1.w;
+                it.q_tok = (int32_t)rec1.x, it.n_tok = (int32_t)rec1.y;
                 if (it.n_tok <= 0) break;
-                const int n_tiles = tiles_of(it);
+                const int n_tiles = (it.key_end - it.key_begin + kTileKeys - 1) / kTileKeys;
                 const int n_x = it.n_tok > tile_tok ? 2 : 1;
                 const int32_t* bt = p.block_table + (int64_t)it.req * p.max_pages + it.key_begin / kPage;
                 for (int j = 0; j < n_tiles && ok; ++j) {
@@ -714,15 +725,12 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                 }
                 __syncwarp();
             };
-            PrefillItem it, nx;
-            bool have = take_item(n_item, it);
+            int n_tiles = 0, n_x = 0, nx_tiles = 0, nx_n_x = 0;
+            bool have = take_shape(n_item, n_tiles, n_x);
             ++n_item;
             bool pre[2] = {false, false};  // S_x of the item's first key tile was issued at the end of the previous item
             while (have && ok) {
-                const int n_tiles = tiles_of(it);
-                const int n_x = it.n_tok > tile_tok ? 2 : 1;
                 bool have_next = false;
-                int nx_tiles = 0, nx_n_x = 0;
                 for (int x = 0; x < n_x && ok; ++x)
                     if (!pre[x]) issue_qk(tile_ctr, x, n_x, true, n_tiles == 1, items_x[x]);
                 pre[0] = pre[1] = false;
@@ -730,12 +738,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                     const uint32_t tc = tile_ctr + j;
                     const uint32_t s = tc & 1;
                     if (j == n_tiles - 1) {
-                        have_next = take_item(n_item, nx);
+                        have_next = take_shape(n_item, nx_tiles, nx_n_x);
                         ++n_item;
-                        if (have_next) {
-                            nx_tiles = tiles_of(nx);
-                            nx_n_x = nx.n_tok > tile_tok ? 2 : 1;
-                        }
                     }
                     for (int x = 0; x < n_x && ok; ++x) {
                         ok = wait_all(bars + Bars::p_ready + 8 * x, (tiles_x[x] + j) & 1, s_abort);
@@ -775,7 +779,8 @@ __global__ void __launch_bounds__(kThreads, 1) prefill_kernel(const PrefillParam
                     tiles_x[x] += n_tiles;
                     ++items_x[x];
                 }
-                it = nx;
+                n_tiles = nx_tiles;
+                n_x = nx_n_x;
                 have = have_next;
             }
         }
