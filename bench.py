@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of one serving iteration's mixed-batch paged-KV attention.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 1|2|4]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 1|2|3|4]
 
 A step is one pass of the whole path over one synthetic batch: host work
 partition (ps_attn_plan), then ps_attn_run (work-list upload, prefill, decode
@@ -61,8 +61,8 @@ def measured_peaks():
 # proportion to the KV a launch reads, so a full launch is the ratio times its algorithmic bytes).  The decode
 # kernel's algorithmic bytes are the KV it streams; for the prefill kernel the ratio is per KV byte of its chunks'
 # sequences (its K/V tiles are re-read from L2, not from DRAM).  Re-captured whenever a kernel changes.
-NCU_TRAFFIC_RATIO = {"decode_kernel": 1.012}
-NCU_TRAFFIC_SOURCE = "profiles/decode_kernel_config1.md"
+NCU_TRAFFIC_RATIO = {"decode_kernel": 1.009}
+NCU_TRAFFIC_SOURCE = "profiles/mixed_step_config2.md"
 
 
 def ncu_traffic(kernel, algorithmic_units):
@@ -619,17 +619,86 @@ def run_ours(args):
     return 0
 
 
+def run_grid(args):
+    """--workload 3: seed 0 of each of the 72 cells of the latency-table grid (the scheduler's profile of section
+    4.5): the GPU latency of one ps_attn_run and, beside it, the seconds the CPU oracle needs for the same cell (run in
+    full while a cell's fp64 work stays under the sample budgets, else on a bounded sample and extrapolated by work)."""
+    import torch
+    import paper_2507_17769_b200 as ps  # noqa: F401
+    from workloads.device import DeviceBatch
+
+    rank, local_rank, world = dist_env()
+    if rank != 0:
+        return 0
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; the library has no CPU path")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    rows, tot_bytes, tot_ms, tot_cpu, threads = [], 0.0, 0.0, 0.0, 1
+    for cell, chunk, nd, m in gen.grid_cells():
+        batch = gen.config3_cell(chunk, nd, m, gen.grid_seed(cell, 0))
+        db = DeviceBatch(batch, poison=False, device=dev)
+        db.plan()
+        out = torch.empty_like(db.q)
+        for _ in range(max(3, args.warmup)):
+            db.pa.run(db.q, db.block_table, out=out, want_lse=False)
+        n = max(5, min(args.steps, 50))
+        torch.cuda.synchronize(dev)
+        ev0.record()
+        for _ in range(n):
+            db.pa.run(db.q, db.block_table, out=out, want_lse=False)
+        ev1.record()
+        torch.cuda.synchronize(dev)
+        db.pa.check()
+        gpu_us = ev0.elapsed_time(ev1) / n * 1e3
+        cpu_s, sampled = float("nan"), 0
+        if not args.no_cpu_baseline:
+            dec, rws = oracle_sample(batch)
+            sampled = int(len(dec) < nd or sum(len(v) for v in rws.values()) < chunk)
+            sample = OracleSample(batch, dec, rws, dev)
+            dt_d, bytes_d, dt_p, flops_p, threads = sample.time()
+            cpu_s = sample.whole_step(dt_d, bytes_d, dt_p, flops_p)
+            tot_cpu += cpu_s
+        rows.append((chunk, nd, m, batch.seed, int(batch.kv_len.sum()), batch.decode_bytes(), batch.prefill_flops(), gpu_us,
+                     cpu_s, sampled, threads))
+        tot_bytes += float(batch.decode_bytes())
+        tot_ms += gpu_us * 1e-3
+        db.pa.close()
+        del db, out
+    if args.grid_csv:
+        with open(args.grid_csv, "w") as f:
+            f.write("chunk,n_decode,mean_ctx,seed,kv_tokens,decode_bytes,prefill_flops,gpu_latency_us,cpu_seconds,cpu_sampled,cpu_cores\n")
+            for r in rows:
+                f.write("%d,%d,%d,%d,%d,%d,%d,%.3f,%.4f,%d,%d\n" % r)
+    line = {"metric": METRIC, "value": tot_bytes / (tot_ms * 1e-3) / 1e12, "unit": "TB/s", "n_gpus": 1, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": tot_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "config3: latency-table grid, seed 0 of each of %d cells (a step = one run of every cell)" % len(rows),
+                       "cells": len(rows), "csv": args.grid_csv},
+            "cpu_baseline": {"value": tot_bytes / tot_cpu / 1e12 if tot_cpu > 0 else None, "unit": "TB/s", "cores": threads,
+                             "kind": "oracle", "seconds_all_cells": tot_cpu,
+                             "sample": "every cell; cells above the sample budgets are timed on a bounded sample and extrapolated"}}
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", type=int, default=4, choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", type=int, default=4, choices=sorted(WORKLOADS) + [3])
+    ap.add_argument("--grid-csv", default=None, help="--workload 3: write one row per grid cell (GPU latency, CPU oracle seconds)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--shard", default="requests", choices=["requests", "heads"],
                     help="what N > 1 ranks split: requests (each rank its own batch; default) or the KV heads of one batch")
     args = ap.parse_args()
+    if args.workload == 3:
+        if args.impl == "reference" or args.gpus != 1:
+            raise SystemExit("--workload 3 (the per-cell grid) runs on one GPU with --impl ours")
+        return run_grid(args)
     if args.impl == "reference":
         args.steps = min(args.steps, 3)  # each step is seconds of CPU work
         return run_reference(args)

@@ -23,6 +23,8 @@ _lib = None
 _I32P = ctypes.POINTER(ctypes.c_int32)
 _U16P = ctypes.POINTER(ctypes.c_uint16)
 _F64P = ctypes.POINTER(ctypes.c_double)
+_U8P = ctypes.POINTER(ctypes.c_uint8)
+_F32P = ctypes.POINTER(ctypes.c_float)
 
 
 def build(force: bool = False) -> str:
@@ -50,6 +52,12 @@ def _load():
         lib.oracle_attn_paged.argtypes = [
             _U16P, _U16P, _U16P, ctypes.c_int64, _I32P, ctypes.c_int32, _I32P, _I32P, ctypes.c_int32,
             ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, _F64P, _F64P,
+        ]
+        lib.oracle_attn_rows_fp8.restype = ctypes.c_int
+        lib.oracle_attn_rows_fp8.argtypes = [
+            _U16P, _U8P, _U8P, _F32P, _F32P, _F64P, ctypes.c_int64, _I32P, ctypes.c_int32, _I32P, _I32P, ctypes.c_int32,
+            ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+            _I32P, _I32P, ctypes.c_int64, _F64P, _F64P,
         ]
         lib.oracle_kv_gather.restype = ctypes.c_int
         lib.oracle_kv_gather.argtypes = [
@@ -104,6 +112,62 @@ def attn_rows(q, k_pool, v_pool, block_table, prior, q_len, n_q_heads, n_kv_head
     if rc != 0:
         raise ValueError("oracle_attn_rows failed with code %d" % rc)
     return out, lse
+
+
+def attn_rows_fp8(q, k_codes, v_codes, k_scale, v_scale, block_table, prior, q_len, n_q_heads, n_kv_heads, head_dim,
+                  page_size, row_req, row_tok):
+    """Oracle attention over an FP8 (E4M3) cache: codes uint8 [pages, page, Hkv, d], scales float32 [pages, page, Hkv]
+    (see ``oracle.fp8``).  Returns (out [R,Hq,d], lse [R,Hq]) float64."""
+    from . import fp8
+
+    lib = _load()
+    q = _c(q, np.uint16)
+    k_codes = _c(k_codes, np.uint8)
+    v_codes = _c(v_codes, np.uint8)
+    k_scale = _c(k_scale, np.float32)
+    v_scale = _c(v_scale, np.float32)
+    block_table = _c(block_table, np.int32)
+    prior = _c(prior, np.int32)
+    q_len = _c(q_len, np.int32)
+    row_req = _c(row_req, np.int32)
+    row_tok = _c(row_tok, np.int32)
+    table = _c(fp8.decode_table(), np.float64)
+    n = prior.shape[0]
+    assert q.shape == (int(q_len.sum()), n_q_heads, head_dim), q.shape
+    assert k_codes.shape[1:] == (page_size, n_kv_heads, head_dim) and v_codes.shape == k_codes.shape
+    assert k_scale.shape == k_codes.shape[:3] and v_scale.shape == k_scale.shape
+    R = row_req.shape[0]
+    out = np.empty((R, n_q_heads, head_dim), dtype=np.float64)
+    lse = np.empty((R, n_q_heads), dtype=np.float64)
+    rc = lib.oracle_attn_rows_fp8(
+        _p(q, _U16P), _p(k_codes, _U8P), _p(v_codes, _U8P), _p(k_scale, _F32P), _p(v_scale, _F32P), _p(table, _F64P),
+        k_codes.shape[0], _p(block_table, _I32P), block_table.shape[1], _p(prior, _I32P), _p(q_len, _I32P), n,
+        n_q_heads, n_kv_heads, head_dim, page_size, _p(row_req, _I32P), _p(row_tok, _I32P), R,
+        _p(out, _F64P), _p(lse, _F64P),
+    )
+    if rc != 0:
+        raise ValueError("oracle_attn_rows_fp8 failed with code %d" % rc)
+    return out, lse
+
+
+def plain_pool_fp8(kv_bits_per_request, block_table, num_pages, page_size):
+    """Quantise logical bf16 tensors (uint16 [kv_len_r, Hkv, d] each) token by token and lay them out in the oracle's
+    paged form: (codes uint8 [pages, page, Hkv, d], scales float32 [pages, page, Hkv]).  Slots nobody references hold
+    the E4M3 NaN code and a NaN scale."""
+    from . import fp8
+
+    hkv, d = kv_bits_per_request[0].shape[1:]
+    codes = np.full((num_pages, page_size, hkv, d), 0x7F, dtype=np.uint8)
+    scales = np.full((num_pages, page_size, hkv), np.nan, dtype=np.float32)
+    for r, x in enumerate(kv_bits_per_request):
+        c, s = fp8.quantise(x)
+        L = x.shape[0]
+        for pi in range((L + page_size - 1) // page_size):
+            lo = pi * page_size
+            hi = min(L, lo + page_size)
+            codes[int(block_table[r, pi]), : hi - lo] = c[lo:hi]
+            scales[int(block_table[r, pi]), : hi - lo] = s[lo:hi]
+    return codes, scales
 
 
 def attn_paged(q, k_pool, v_pool, block_table, prior, q_len, n_q_heads, n_kv_heads, head_dim, page_size):

@@ -32,7 +32,8 @@
  * in extended precision, constant V, single key, one-hot key, zero Q (prefix
  * mean), chunk split == unchunked, decode row == last prefill row, key
  * permutation invariance, GQA mapping, torch CPU fp64 causal SDPA, page
- * permutation with NaN-poisoned spare pages, split + log-sum-exp merge.
+ * permutation with NaN-poisoned spare pages, split + log-sum-exp merge; the FP8
+ * variant equals the bf16 one on data that E4M3 holds exactly.
  */
 #include <math.h>
 #include <stdint.h>
@@ -133,6 +134,99 @@ int oracle_attn_rows(const uint16_t *q, const uint16_t *k_pool, const uint16_t *
                 const uint16_t *vv = v_pool + ((page * page_size + j % page_size) * Hkv + g) * (int64_t)d;
                 const double p = s[j] / denom;
                 for (int t = 0; t < d; ++t) o[t] += p * bf16_to_f64(vv[t]);
+            }
+            lse[k * Hq + h] = m + log(denom);
+        }
+        free(s);
+    }
+    free(q_start);
+    return bad ? -6 : 0;
+}
+
+/*
+ * The same attention over an FP8 (E4M3) KV cache: k_codes / v_codes hold one code per element,
+ * uint8 [num_pages][page_size][Hkv][d]; k_scale / v_scale one fp32 scale per (token, kv head),
+ * float [num_pages][page_size][Hkv]; an element's value is e4m3[code] * scale, evaluated in fp64
+ * (exact).  e4m3 is the 256-entry table of code values (built by the caller from the format's
+ * definition: bias 7, 3 mantissa bits, subnormals m * 2^-9).  Q stays bf16.  The quantisation
+ * format is this repository's reading (the paper states no precision); the arithmetic below is
+ * the plain definition again.
+ */
+int oracle_attn_rows_fp8(const uint16_t *q, const uint8_t *k_codes, const uint8_t *v_codes,
+                         const float *k_scale, const float *v_scale, const double *e4m3,
+                         int64_t num_pages, const int32_t *block_table, int32_t max_pages,
+                         const int32_t *prior, const int32_t *q_len, int32_t n,
+                         int32_t Hq, int32_t Hkv, int32_t d, int32_t page_size,
+                         const int32_t *row_req, const int32_t *row_tok, int64_t n_rows,
+                         double *out, double *lse) {
+    if (Hq <= 0 || Hkv <= 0 || Hq % Hkv != 0 || d <= 0 || page_size <= 0) return -1;
+    const int G = Hq / Hkv;
+    int64_t *q_start = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));
+    if (!q_start) return -2;
+    q_start[0] = 0;
+    for (int r = 0; r < n; ++r) {
+        if (q_len[r] < 1 || prior[r] < 0) { free(q_start); return -3; }
+        if ((int64_t)prior[r] + q_len[r] > (int64_t)max_pages * page_size) { free(q_start); return -4; }
+        q_start[r + 1] = q_start[r] + q_len[r];
+    }
+    for (int64_t k = 0; k < n_rows; ++k) {
+        int r = row_req[k];
+        if (r < 0 || r >= n || row_tok[k] < 0 || row_tok[k] >= q_len[r]) { free(q_start); return -5; }
+    }
+    int bad = 0;
+    const double scale = 1.0 / sqrt((double)d);
+    const int64_t n_work = n_rows * Hq;
+#pragma omp parallel
+    {
+        double *s = NULL;
+        int64_t cap = 0;
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t w = 0; w < n_work; ++w) {
+            const int64_t k = w / Hq;
+            const int h = (int)(w % Hq);
+            const int g = h / G;
+            const int r = row_req[k];
+            const int i = row_tok[k];
+            const int64_t L = (int64_t)prior[r] + i + 1;
+            if (L > cap) {
+                free(s);
+                s = (double *)malloc(sizeof(double) * (size_t)L);
+                cap = L;
+            }
+            const uint16_t *qv = q + ((q_start[r] + i) * Hq + h) * (int64_t)d;
+            const int32_t *bt = block_table + (int64_t)r * max_pages;
+            /* scores */
+            for (int64_t j = 0; j < L; ++j) {
+                const int64_t page = bt[j / page_size];
+                if (page < 0 || page >= num_pages) {
+#pragma omp atomic write
+                    bad = 1;
+                    s[j] = 0.0;
+                    continue;
+                }
+                const int64_t slot = (page * page_size + j % page_size) * Hkv + g;
+                const uint8_t *kc = k_codes + slot * (int64_t)d;
+                const double ks = (double)k_scale[slot];
+                double acc = 0.0;
+                for (int t = 0; t < d; ++t) acc += bf16_to_f64(qv[t]) * (e4m3[kc[t]] * ks);
+                s[j] = acc * scale;
+            }
+            /* softmax by max subtraction */
+            double m = s[0];
+            for (int64_t j = 1; j < L; ++j) if (s[j] > m) m = s[j];
+            double denom = 0.0;
+            for (int64_t j = 0; j < L; ++j) { s[j] = exp(s[j] - m); denom += s[j]; }
+            /* weighted sum of V */
+            double *o = out + (k * Hq + h) * (int64_t)d;
+            for (int t = 0; t < d; ++t) o[t] = 0.0;
+            for (int64_t j = 0; j < L; ++j) {
+                const int64_t page = bt[j / page_size];
+                if (page < 0 || page >= num_pages) continue;
+                const int64_t slot = (page * page_size + j % page_size) * Hkv + g;
+                const uint8_t *vc = v_codes + slot * (int64_t)d;
+                const double vs = (double)v_scale[slot];
+                const double p = s[j] / denom;
+                for (int t = 0; t < d; ++t) o[t] += p * (e4m3[vc[t]] * vs);
             }
             lse[k * Hq + h] = m + log(denom);
         }

@@ -170,7 +170,7 @@ def peak_kv(kv_len, remaining):
     """(largest total KV-cache size over the future iterations, first iteration where it occurs)."""
     peak, when = 0, 0
     horizon = max(remaining) if len(remaining) else 0
-    for t in range(horizon):  # "simulates future iterations ... and exits when finished"
+    for t in range(horizon):  # admission look-ahead (section 4.5): step iteration by iteration until every request is done
         kv, _ = kv_at(kv_len, remaining, t)
         if kv > peak:
             peak, when = kv, t

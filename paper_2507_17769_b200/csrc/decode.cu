@@ -26,15 +26,10 @@ namespace ps {
 
 namespace {
 
-#ifndef PS_DECODE_WARPS
-#define PS_DECODE_WARPS 12
-#endif
-#ifndef PS_DECODE_STAGES
-#define PS_DECODE_STAGES 2
-#endif
 // streaming warps per CTA (one CTA per SM) and ring depth per warp: 12 x 2 x 8 KB = 192 KB in flight per SM;
 // measured on B200: 12 x 2 and 10 x 2 beat 8 x 3, 6 x 4 and 4 x 6 by 2-6 %
-constexpr int kWarps = PS_DECODE_WARPS;
+constexpr int kWarps = 12;
+constexpr int kStagesPerWarp = 2;
 constexpr int kRing = 8;  // unit ids in flight between the producer and consumer cursors of a warp
 constexpr int kDeferred = 8;  // merges a warp can postpone until its KV stream has drained
 
@@ -42,7 +37,7 @@ template <int D>
 struct DecodeCfg {
     static constexpr int kBlockBytes = kPage * D * 2;      // K (or V) of one page, one kv head
     static constexpr int kStageBytes = 2 * kBlockBytes;    // K then V
-    static constexpr int kStages = (D == 128) ? PS_DECODE_STAGES : 2 * PS_DECODE_STAGES;  // 8 KB (4 KB) stages per warp
+    static constexpr int kStages = (D == 128) ? kStagesPerWarp : 2 * kStagesPerWarp;  // 8 KB (4 KB) stages per warp
     static constexpr int kSmemBytes =
         kWarps * kStages * kStageBytes + kWarps * kStages * 8 + kWarps * kRing * 4 + kWarps * kDeferred * 12 + 1024;
 };

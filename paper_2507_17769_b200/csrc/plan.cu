@@ -22,10 +22,7 @@ namespace ps {
 
 static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-#ifndef PS_DECODE_UNITS_PER_WARP
-#define PS_DECODE_UNITS_PER_WARP 1
-#endif
-constexpr int kDecodeUnitsPerWarp = PS_DECODE_UNITS_PER_WARP;  // work units per resident warp (measured: 1 beats 2 and 3 on the decode-only batch)
+constexpr int kDecodeUnitsPerWarp = 1;  // work units per resident warp (measured: 1 beats 2 and 3 on the decode-only batch)
 // Smallest decode unit (pages) of a batch too small to give every warp its share: between 4 and 8, so that the
 // longest row is cut into about 16 pieces at most.  Finer cuts spread a small batch over more warps (64 rows of
 // 64 tokens: 13 us instead of 20; 8 rows of 512: 16 instead of 23), but every further piece of a row is one more
@@ -34,18 +31,9 @@ constexpr int kDecodeMinPagesLo = 4, kDecodeMinPagesHi = 8, kDecodePiecesPerRow 
 constexpr int kPrefillKeyTile = 128;    // keys per tensor-core tile
 // Measured on B200 (decode: bandwidth against the number of SMs the kernel runs on; prefill: time of one
 // key-tile step of a q tile pair), used to split the SMs of a mixed batch between the two kernels.
-#ifndef PS_DECODE_PEAK
-#define PS_DECODE_PEAK 6.7e12
-#endif
-#ifndef PS_DECODE_SHARED_PEAK
-#define PS_DECODE_SHARED_PEAK 6.0e12
-#endif
-#ifndef PS_DECODE_PER_SM
-#define PS_DECODE_PER_SM 115e9
-#endif
-constexpr double kDecodePeakBytesPerSec = PS_DECODE_PEAK;
-constexpr double kDecodeSharedPeakBytesPerSec = PS_DECODE_SHARED_PEAK;  // decode rows beside a running prefill kernel
-constexpr double kDecodeBytesPerSecPerSm = PS_DECODE_PER_SM;
+constexpr double kDecodePeakBytesPerSec = 6.7e12;
+constexpr double kDecodeSharedPeakBytesPerSec = 6.0e12;  // decode rows beside a running prefill kernel
+constexpr double kDecodeBytesPerSecPerSm = 115e9;
 constexpr double kDecodeAloneBytesPerSecPerSm = 135e9;  // per SM with the memory system to itself
 constexpr double kPrefillStepSec = 2.5e-6;
 constexpr double kKernelFloorSec = 12e-6;
@@ -208,43 +196,43 @@ static void plan_decode(ps_plan* pl, const int32_t* prior, const int32_t* q_len,
     for (int r = 0; r < pl->n; ++r) {
         if (!runs_as_decode(pl->shape, pl->tiny_as_rows, prior[r], q_len[r])) continue;
         for (int i = 0; i < q_len[r]; ++i) {  // one row per new token (a decode request has one)
-        const int kv_len = prior[r] + i + 1;
-        const int pages = (kv_len + kPage - 1) / kPage;
-        const int32_t q_tok = q_start[r] + i;
-        for (int g = 0; g < Hkv; ++g) {
-            const int32_t first_piece = n_pieces;
-            int pg = 0;
-            while (pg < pages) {
-                if (room == 0) {
-                    if (n_units > 0) units[n_units - 1].piece_end = n_pieces;
-                    units[n_units++].piece_begin = n_pieces;
-                    room = per_unit;
+            const int kv_len = prior[r] + i + 1;
+            const int pages = (kv_len + kPage - 1) / kPage;
+            const int32_t q_tok = q_start[r] + i;
+            for (int g = 0; g < Hkv; ++g) {
+                const int32_t first_piece = n_pieces;
+                int pg = 0;
+                while (pg < pages) {
+                    if (room == 0) {
+                        if (n_units > 0) units[n_units - 1].piece_end = n_pieces;
+                        units[n_units++].piece_begin = n_pieces;
+                        room = per_unit;
+                    }
+                    const int take = (int)std::min<int64_t>(room, pages - pg);
+                    DecodePiece& pc = pieces[n_pieces++];
+                    pc.req = r;
+                    pc.kv_head = g;
+                    pc.page_begin = pg;
+                    pc.page_end = pg + take;
+                    pc.q_tok = q_tok;
+                    pc.part_slot = -1;
+                    pc.kv_len = kv_len;
+                    pc.merge_idx = 0;
+                    pg += take;
+                    room -= take;
                 }
-                const int take = (int)std::min<int64_t>(room, pages - pg);
-                DecodePiece& pc = pieces[n_pieces++];
-                pc.req = r;
-                pc.kv_head = g;
-                pc.page_begin = pg;
-                pc.page_end = pg + take;
-                pc.q_tok = q_tok;
-                pc.part_slot = -1;
-                pc.kv_len = kv_len;
-                pc.merge_idx = 0;
-                pg += take;
-                room -= take;
-            }
-            const int32_t cnt = n_pieces - first_piece;
-            if (cnt > 1) {
-                for (int32_t s = 0; s < cnt; ++s) {
-                    pieces[first_piece + s].part_slot = (int32_t)(slots + (int64_t)s * G);
-                    pieces[first_piece + s].merge_idx = n_dmerge;
+                const int32_t cnt = n_pieces - first_piece;
+                if (cnt > 1) {
+                    for (int32_t s = 0; s < cnt; ++s) {
+                        pieces[first_piece + s].part_slot = (int32_t)(slots + (int64_t)s * G);
+                        pieces[first_piece + s].merge_idx = n_dmerge;
+                    }
+                    dmerge[n_dmerge].base = (int32_t)slots;
+                    dmerge[n_dmerge].n_seg = cnt;
+                    ++n_dmerge;
+                    slots += (int64_t)cnt * G;
                 }
-                dmerge[n_dmerge].base = (int32_t)slots;
-                dmerge[n_dmerge].n_seg = cnt;
-                ++n_dmerge;
-                slots += (int64_t)cnt * G;
             }
-        }
         }
     }
     if (n_units > 0) units[n_units - 1].piece_end = n_pieces;
