@@ -424,7 +424,10 @@ def run_ours(args):
     desc, make, seed = WORKLOADS[args.workload]
     batch = shard_batch(make, seed, rank, world, args.shard)
     s = batch.shape
-    db = DeviceBatch(batch, poison=False, device=dev)
+    fp8 = args.kv_cache == "fp8"
+    if fp8 and float(batch.prefill_flops()) > 0:
+        raise SystemExit("--kv-cache fp8: the FP8 cache variant serves decode rows only (use --workload 1)")
+    db = DeviceBatch(batch, poison=False, device=dev, kv_dtype=1 if fp8 else 0)
     pa = db.pa
     info = db.plan()
     stream = torch.cuda.current_stream(dev)
@@ -471,6 +474,8 @@ def run_ours(args):
         ps.ps_plan_set_timing(pa._plan, 0)
     pa.check()
     dec_bytes, pf_flops = float(batch.decode_bytes()), float(batch.prefill_flops())
+    if fp8:  # one byte per element plus an fp32 scale per (token, kv head) for K and for V
+        dec_bytes = float(batch.decode_kv_tokens()) * (2 * s.n_kv_heads * s.head_dim + 2 * s.n_kv_heads * 4)
     ms, units = reduce_over_ranks(local_ms, dec_bytes, world, dev)
     value = units / (ms * 1e-3) / 1e12
 
@@ -573,7 +578,7 @@ def run_ours(args):
         if t_hbm >= t_tensor:
             ach = dec_bytes / (ms * 1e-3) / 1e9
             roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                    "traffic": ncu_traffic("decode_kernel", dec_bytes), "dominant_kernel": "decode_kernel"}
+                    "traffic": None if fp8 else ncu_traffic("decode_kernel", dec_bytes), "dominant_kernel": "decode_kernel"}
         else:
             ach = pf_flops / (ms * 1e-3) / 1e12
             roof = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
@@ -587,7 +592,8 @@ def run_ours(args):
             "metric": METRIC, "value": value, "unit": "TB/s", "n_gpus": world, "steps": args.steps, "warmup": warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "strong" if args.shard == "heads" and world > 1 else "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": desc, "kv_bytes_per_step_per_gpu": dec_bytes, "prefill_flops_per_step_per_gpu": pf_flops,
+            "config": {"workload": desc + (" [KV cache in FP8 E4M3 with per-token scales]" if fp8 else ""),
+                       "kv_cache": args.kv_cache, "kv_bytes_per_step_per_gpu": dec_bytes, "prefill_flops_per_step_per_gpu": pf_flops,
                        "l2": "inputs larger than L2 (%.0f MB of KV per step), no flush" % (dec_bytes / 1e6),
                        "decode_items": info.n_decode_items, "prefill_items": info.n_prefill_items,
                        "merge_rows": info.n_merge_rows, "decode_sms": info.decode_sms, "prefill_sms": info.prefill_sms,
@@ -606,7 +612,7 @@ def run_ours(args):
             "roofline": roof,
         }
         # ---- CPU baseline: the oracle as it stands, on the host's cores, on a bounded sample ----
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and not fp8:
             dec, rows = oracle_sample(batch)
             sample = OracleSample(batch, dec, rows, dev)
             line["cpu_baseline"] = cpu_baseline_record(batch, sample, sample.time())
@@ -692,6 +698,9 @@ def main():
     ap.add_argument("--workload", type=int, default=4, choices=sorted(WORKLOADS) + [3])
     ap.add_argument("--grid-csv", default=None, help="--workload 3: write one row per grid cell (GPU latency, CPU oracle seconds)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kv-cache", default="bf16", choices=["bf16", "fp8"],
+                    help="fp8: the E4M3 cache variant of the decode path (decode-only workloads; bytes counted at one per "
+                         "element plus the scales)")
     ap.add_argument("--shard", default="requests", choices=["requests", "heads"],
                     help="what N > 1 ranks split: requests (each rank its own batch; default) or the KV heads of one batch")
     args = ap.parse_args()

@@ -48,8 +48,20 @@ typedef enum {
 } ps_status;
 
 /* Attention geometry.  Supported: head_dim in {64, 128}, page_size == 16,
- * n_q_heads a multiple of n_kv_heads, dtype == 0 (bf16 in, fp32 accumulate,
- * bf16 out). */
+ * n_q_heads a multiple of n_kv_heads (1, 2, 4 or 8 q heads per kv head).
+ * dtype == 0: bf16 K/V cache (bf16 in, fp32 accumulate, bf16 out).
+ * dtype == 1: the cache holds K and V as FP8 E4M3 codes with one fp32 scale per
+ * (token, kv head) and tensor -- scale = amax / 448 over the head_dim values,
+ * rounded up to 8 significant bits (1 for an all-zero vector), code = x /
+ * scale rounded to nearest even and
+ * saturated at +-448, both divisions IEEE fp32; a stored token never changes
+ * when later tokens are appended.  Q and out stay bf16, accumulation fp32; the
+ * decode kernel multiplies with f16 operands (E4M3 converts to f16 exactly), so
+ * Q is clamped to +-65504 and V scales are meant to lie in [2.4e-7, 255].  The
+ * paper states no precision (its section 3.3 only notes that decode attention
+ * time is set by the bytes of KV cache read); this variant halves those bytes.
+ * It exists for head_dim 128 and serves decode rows only: ps_attn_plan refuses
+ * batches with q_len > 1 and ps_profile_grid sweeps the bf16 cache only. */
 typedef struct {
     int32_t n_q_heads;
     int32_t n_kv_heads;
@@ -111,6 +123,17 @@ ps_status ps_kv_write(ps_kv *kv, const void *k_new_dev, const void *v_new_dev, c
  */
 ps_status ps_kv_gather(const ps_kv *kv, const int32_t *block_table_row_dev, int32_t len, void *k_out_dev,
                        void *v_out_dev, void *stream);
+
+/*
+ * FP8 pools (dtype == 1): ps_kv_write takes the same bf16 inputs and quantises
+ * them as ps_shape describes; ps_kv_gather returns the codes, one byte per
+ * element ([len, n_kv_heads, head_dim] uint8 in k_out_dev / v_out_dev).
+ * ps_kv_gather_fp8 returns codes and the fp32 scales ([len, n_kv_heads]); any
+ * output may be NULL.  Together they let a test compare the stored cache bit
+ * for bit with a reference quantiser.  PS_ERR_INVALID on a bf16 pool.
+ */
+ps_status ps_kv_gather_fp8(const ps_kv *kv, const int32_t *block_table_row_dev, int32_t len, void *k_codes_out_dev,
+                           void *v_codes_out_dev, float *k_scale_out_dev, float *v_scale_out_dev, void *stream);
 
 /* Synchronises `stream`, then returns PS_OK or PS_ERR_BOUNDS for the pool's
  * write/gather kernels since the last call, and clears the flag. */

@@ -5,9 +5,14 @@ The library's FP8 cache variant stores K and V as OCP FP8 E4M3 codes (1 sign,
 infinities; S.1111.111 is NaN) with one fp32 scale per (token, kv head) and
 tensor:
 
-    scale = amax / 448        amax = max |x| over the head_dim values (scale = 1 if amax = 0)
+    scale = amax / 448 rounded up to 8 significant bits (a bf16-representable fp32)
+            amax = max |x| over the head_dim values (scale = 1 if amax = 0)
     code  = round_to_nearest_even_e4m3( x / scale ), saturating at +-448
     value = decode(code) * scale
+
+(The scale keeps 8 significant bits so that a softmax weight of exactly 1 times
+the scale is still exact in a 16-bit matrix operand; rounding up keeps
+|x| / scale <= 448.)
 
 The paper states no precision; this format is this repository's reading.  The
 divisions are IEEE fp32 (both sides take the rounding decision in that
@@ -76,6 +81,9 @@ def quantise(x_bits: np.ndarray):
     x = u.view(np.float32)
     amax = np.max(np.abs(x), axis=-1)
     scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    u = scale.view(np.uint32)
+    u = np.where((u & np.uint32(0xFFFF)) != 0, (u | np.uint32(0xFFFF)) + np.uint32(1), u).astype(np.uint32)  # round up to bf16 precision
+    scale = u.view(np.float32)
     y = (x / scale[..., None]).astype(np.float32)  # IEEE fp32 division
     return encode(y), scale
 

@@ -7,7 +7,7 @@ wrapper that keeps the pool, plan and workspace of one engine together.
 All arithmetic runs in the CUDA kernels; there is no CPU path.
 """
 from .binding import (  # noqa: F401
-    PS_STATIC_WORKSPACE_BYTES, PsError, make_shape, ps_attn_plan, ps_attn_run, ps_attn_run_static, ps_grid_row, ps_kv_alloc, ps_kv_bytes, ps_kv_free, ps_kv_gather,
+    PS_STATIC_WORKSPACE_BYTES, PsError, make_shape, ps_attn_plan, ps_attn_run, ps_attn_run_static, ps_grid_row, ps_kv_alloc, ps_kv_bytes, ps_kv_free, ps_kv_gather, ps_kv_gather_fp8,
     ps_kv_status, ps_kv_write, ps_last_error, ps_plan_free, ps_plan_get_info, ps_plan_get_items, ps_plan_info,
     ps_plan_get_timing, ps_plan_opts, ps_plan_set_timing, ps_plan_set_wait_limit, ps_plan_status, ps_profile_grid, ps_shape, ps_version,
 )

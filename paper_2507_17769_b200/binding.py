@@ -64,7 +64,7 @@ class ps_grid_row(ctypes.Structure):
                 ("prefill_TFLOPs", ctypes.c_float), ("roofline_frac", ctypes.c_float)]
 
 
-EXPORTS = ["ps_kv_bytes", "ps_kv_alloc", "ps_kv_free", "ps_kv_write", "ps_kv_gather", "ps_kv_status", "ps_attn_plan",
+EXPORTS = ["ps_kv_bytes", "ps_kv_alloc", "ps_kv_free", "ps_kv_write", "ps_kv_gather", "ps_kv_gather_fp8", "ps_kv_status", "ps_attn_plan",
            "ps_plan_free", "ps_plan_get_info", "ps_plan_get_items", "ps_attn_run", "ps_plan_status",
            "ps_plan_set_timing", "ps_plan_get_timing", "ps_plan_set_wait_limit", "ps_profile_grid", "ps_attn_run_static",
            "ps_last_error", "ps_version"]
@@ -89,6 +89,7 @@ def load() -> ctypes.CDLL:
     lib.ps_kv_free.argtypes = [_vp]
     lib.ps_kv_write.argtypes = [_vp, _vp, _vp, _vp, _i32, _i32p, _i32p, _i32, _vp]
     lib.ps_kv_gather.argtypes = [_vp, _vp, _i32, _vp, _vp, _vp]
+    lib.ps_kv_gather_fp8.argtypes = [_vp, _vp, _i32, _vp, _vp, _vp, _vp, _vp]
     lib.ps_kv_status.argtypes = [_vp, _vp]
     lib.ps_attn_plan.argtypes = [sp, _i32p, _i32p, _i32, _i32, ctypes.POINTER(ps_plan_opts), ctypes.POINTER(_vp),
                                  ctypes.POINTER(_sz)]
@@ -170,6 +171,11 @@ def ps_kv_write(kv, k_new_dev, v_new_dev, block_table_dev, max_pages, prior_host
 
 def ps_kv_gather(kv, block_table_row_dev, length, k_out_dev, v_out_dev, stream=None):
     _check(load().ps_kv_gather(kv, _ptr(block_table_row_dev), length, _ptr(k_out_dev), _ptr(v_out_dev), _ptr(stream)))
+
+
+def ps_kv_gather_fp8(kv, block_table_row_dev, length, k_codes_out_dev, v_codes_out_dev, k_scale_out_dev, v_scale_out_dev, stream=None):
+    _check(load().ps_kv_gather_fp8(kv, _ptr(block_table_row_dev), length, _ptr(k_codes_out_dev), _ptr(v_codes_out_dev),
+                                   _ptr(k_scale_out_dev), _ptr(v_scale_out_dev), _ptr(stream)))
 
 
 def ps_kv_status(kv, stream=None):

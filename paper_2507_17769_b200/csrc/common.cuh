@@ -68,6 +68,9 @@ constexpr int kPage = 16;
 
 __host__ __device__ inline size_t block_bytes(int d) { return (size_t)kPage * d * 2; }
 __host__ __device__ inline size_t page_head_bytes(int d) { return 2 * block_bytes(d); }
+// FP8 (E4M3) cache variant: K codes, V codes (16 tokens x d bytes each, rows swizzled by 16-byte unit like a bf16
+// half), then the 16 tokens' K scales and their V scales (fp32)
+__host__ __device__ constexpr size_t fp8_page_head_bytes(int d) { return 2 * (size_t)kPage * d + 2 * kPage * sizeof(float); }
 
 // byte offset of the 16-byte unit holding elements [8u', 8u'+8) of token t,
 // where e = element index in [0, d), inside a K or V block

@@ -33,14 +33,42 @@ constexpr int kStagesPerWarp = 2;
 constexpr int kRing = 8;  // unit ids in flight between the producer and consumer cursors of a warp
 constexpr int kDeferred = 8;  // merges a warp can postpone until its KV stream has drained
 
-template <int D>
+// FP8 = the E4M3 cache variant: a (page, kv head) block is K codes, V codes (one byte per element, rows of D bytes
+// with the same 16-byte-unit swizzle), then the 16 tokens' K scales and V scales (fp32).
+template <int D, bool FP8>
 struct DecodeCfg {
-    static constexpr int kBlockBytes = kPage * D * 2;      // K (or V) of one page, one kv head
-    static constexpr int kStageBytes = 2 * kBlockBytes;    // K then V
-    static constexpr int kStages = (D == 128) ? kStagesPerWarp : 2 * kStagesPerWarp;  // 8 KB (4 KB) stages per warp
+    static constexpr int kBlockBytes = FP8 ? kPage * D : kPage * D * 2;                  // K (or V) of one page, one kv head
+    static constexpr int kStageBytes = FP8 ? (int)fp8_page_head_bytes(D) : 2 * kBlockBytes;  // K then V (then the scales)
+    // 8 KB (4 KB at D = 64) stages per warp; the FP8 blocks are half as large, so twice as many are kept in flight
+    static constexpr int kStages = (FP8 ? 2 : 1) * ((D == 128) ? kStagesPerWarp : 2 * kStagesPerWarp);
     static constexpr int kSmemBytes =
         kWarps * kStages * kStageBytes + kWarps * kStages * 8 + kWarps * kRing * 4 + kWarps * kDeferred * 12 + 1024;
 };
+
+// The FP8 variant feeds the warp MMA with f16 operands: an E4M3 code converts to f16 exactly in one instruction
+// (every E4M3 value, subnormals included, is a normal f16 or zero), where a conversion to bf16 would cost the ALU
+// pipe four -- and with them the kernel its memory-bound rate.  Q (bf16) is converted once per row, clamped to the
+// f16 range; a softmax weight times its key's V scale is carried as f16 after a multiplication by 2^8 (taken back
+// out with the row sum), which keeps weights down to 2^-22 / scale out of f16's subnormals.
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes) {
+    uint32_t h;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h) : "h"((unsigned short)two_codes));
+    return h;
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    uint32_t h;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(h) : "f"(fminf(fmaxf(hi, -65504.f), 65504.f)), "f"(fminf(fmaxf(lo, -65504.f), 65504.f)));
+    return h;
+}
+// D(16x8, fp32) += A(16x16, f16, row) * B(16x8, f16, col)
+__device__ __forceinline__ void mma_16816_f16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                              uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+constexpr float kWeightScale = 256.f;  // 2^8, see above
 
 struct DecodeParams {
     const char* pool;
@@ -72,9 +100,9 @@ __device__ __forceinline__ bool piece_pages_ok(const int4& a, const DecodeParams
     return (uint32_t)a.x < (uint32_t)p.n_req && (uint32_t)a.y < (uint32_t)p.Hkv && a.z >= 0 && a.z < a.w && a.w <= p.max_pages;
 }
 
-template <int D>
+template <int D, bool FP8>
 __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodeParams p) {
-    using Cfg = DecodeCfg<D>;
+    using Cfg = DecodeCfg<D, FP8>;
     constexpr int STAGES = Cfg::kStages;
     constexpr int KS = D / 16;  // k-steps of QK^T == m-tiles of PV
 
@@ -262,23 +290,27 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
         l1 += __shfl_xor_sync(0xffffffffu, l1, 8);
         l0 += __shfl_xor_sync(0xffffffffu, l0, 16);
         l1 += __shfl_xor_sync(0xffffffffu, l1, 16);
-        const float inv0 = 1.f / l0, inv1 = 1.f / l1;
+        // (FP8: the accumulators hold the outputs times kWeightScale)
+        const float inv0 = (FP8 ? 1.f / kWeightScale : 1.f) / l0, inv1 = (FP8 ? 1.f / kWeightScale : 1.f) / l1;
         const float lse0 = (m0 + log2f(l0)) * 0.6931471805599453f;
         const float lse1 = (m1 + log2f(l1)) * 0.6931471805599453f;
         const int h_base = C_g * p.G;
+        // accumulator rows `row` and `row + 8` of m-tile mt hold d = 16 mt + row and + 8 -- in the FP8 variant, whose
+        // transposed V fragments pair neighbouring bytes, d = 16 mt + 2 row and the next one
+        constexpr int kRowStep = FP8 ? 2 : 1, kPairStep = FP8 ? 1 : 8;
         if (C_slot < 0) {
             __nv_bfloat16* o0 = p.out + ((int64_t)C_qtok * p.Hq + h_base + col) * D;
             __nv_bfloat16* o1 = o0 + D;
 #pragma unroll
             for (int mt = 0; mt < KS; ++mt) {
-                const int dd = mt * 16 + row;
+                const int dd = mt * 16 + kRowStep * row;
                 if (col < p.G) {
                     o0[dd] = __float2bfloat16_rn(o[mt][0] * inv0);
-                    o0[dd + 8] = __float2bfloat16_rn(o[mt][2] * inv0);
+                    o0[dd + kPairStep] = __float2bfloat16_rn(o[mt][2] * inv0);
                 }
                 if (col + 1 < p.G) {
                     o1[dd] = __float2bfloat16_rn(o[mt][1] * inv1);
-                    o1[dd + 8] = __float2bfloat16_rn(o[mt][3] * inv1);
+                    o1[dd + kPairStep] = __float2bfloat16_rn(o[mt][3] * inv1);
                 }
             }
             if (p.lse && row == 0) {
@@ -290,14 +322,14 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
             float* o1 = o0 + D;
 #pragma unroll
             for (int mt = 0; mt < KS; ++mt) {
-                const int dd = mt * 16 + row;
+                const int dd = mt * 16 + kRowStep * row;
                 if (col < p.G) {
                     o0[dd] = o[mt][0] * inv0;
-                    o0[dd + 8] = o[mt][2] * inv0;
+                    o0[dd + kPairStep] = o[mt][2] * inv0;
                 }
                 if (col + 1 < p.G) {
                     o1[dd] = o[mt][1] * inv1;
-                    o1[dd + 8] = o[mt][3] * inv1;
+                    o1[dd + kPairStep] = o[mt][3] * inv1;
                 }
             }
             if (row == 0) {
@@ -380,8 +412,15 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
             const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q + ((int64_t)C_qtok * p.Hq + C_g * p.G + hh) * D);
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
-                qb[ks][0] = hh < p.G ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
-                qb[ks][1] = hh < p.G ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
+                if constexpr (FP8) {  // k-step ks covers d = 16 ks + 4 (lane % 4) + {0, 1 | 2, 3}: the order of the K bytes a thread gets
+                    const uint32_t w0 = hh < p.G ? __ldg(qrow + ks * 8 + 2 * (lane & 3)) : 0u;
+                    const uint32_t w1 = hh < p.G ? __ldg(qrow + ks * 8 + 2 * (lane & 3) + 1) : 0u;
+                    qb[ks][0] = pack_f16(bf16_lo(w0), bf16_hi(w0));
+                    qb[ks][1] = pack_f16(bf16_lo(w1), bf16_hi(w1));
+                } else {
+                    qb[ks][0] = hh < p.G ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
+                    qb[ks][1] = hh < p.G ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
+                }
             }
 #pragma unroll
             for (int mt = 0; mt < KS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
@@ -403,8 +442,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
             // Slots past the sequence end hold whatever the pool holds (possibly NaN):
             // zero those V rows so that 0 * V stays 0; their scores are masked below.
             char* vb = my_stages + stage * Cfg::kStageBytes + Cfg::kBlockBytes;
-            const int units = (kPage - nvalid) * 8;  // 16-byte units per half
-            for (int h = 0; h < D / 64; ++h)
+            const int units = (kPage - nvalid) * 8;  // 16-byte units per region of 16 rows x 128 bytes
+            for (int h = 0; h < Cfg::kBlockBytes / 2048; ++h)
                 for (int u = lane; u < units; u += 32)
                     *reinterpret_cast<uint4*>(vb + h * 2048 + nvalid * 128 + u * 16) = make_uint4(0, 0, 0, 0);
             fence_proxy_async_smem();  // order these generic writes before the stage's next bulk copy
@@ -413,16 +452,40 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
 
         // S^T = K Q^T : 16 tokens x 8 head columns
         float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+        float x0, x1, x2, x3;
+        float sv_lo = 1.f, sv_hi = 1.f;  // FP8: V scales of this thread's two token rows
+        if constexpr (FP8) {
+            // One ldmatrix brings 16 tokens x 32 bytes: the thread gets bytes d = 16 u + 4 (lane % 4) + {0..3} of rows
+            // `row` and `row + 8` for two 16-byte chunks u, each of which is one k-step after conversion.
 #pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            const uint32_t unit = (uint32_t)(((ks * 2 + (mi >> 1)) & 7) ^ l7);
-            uint32_t a0, a1, a2, a3;
-            ldsm_x4(kbase + (ks >> 2) * 2048 + k_tok_off + (unit << 4), a0, a1, a2, a3);
-            if (ks & 1) mma_16816(sb, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
-            else mma_16816(sa, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+            for (int kp = 0; kp < KS / 2; ++kp) {
+                const uint32_t unit = (uint32_t)(((kp * 2 + (mi >> 1)) & 7) ^ l7);
+                uint32_t r0, r1, r2, r3;
+                ldsm_x4(kbase + k_tok_off + (unit << 4), r0, r1, r2, r3);
+                mma_16816_f16(sa, e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r1), e4m3x2_to_f16x2(r0 >> 16), e4m3x2_to_f16x2(r1 >> 16),
+                              qb[2 * kp][0], qb[2 * kp][1]);
+                mma_16816_f16(sb, e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r3), e4m3x2_to_f16x2(r2 >> 16), e4m3x2_to_f16x2(r3 >> 16),
+                              qb[2 * kp + 1][0], qb[2 * kp + 1][1]);
+            }
+            const float* scales = reinterpret_cast<const float*>(my_stages + stage * Cfg::kStageBytes + 2 * Cfg::kBlockBytes);
+            const float fk_lo = scales[row] * p.scale_log2, fk_hi = scales[row + 8] * p.scale_log2;
+            x0 = (sa[0] + sb[0]) * fk_lo, x1 = (sa[1] + sb[1]) * fk_lo;
+            x2 = (sa[2] + sb[2]) * fk_hi, x3 = (sa[3] + sb[3]) * fk_hi;
+            // slots past the sequence end hold arbitrary scales: their weights are zero, keep 0 * scale = 0
+            sv_lo = row < nvalid ? scales[kPage + row] * kWeightScale : 0.f;
+            sv_hi = row + 8 < nvalid ? scales[kPage + row + 8] * kWeightScale : 0.f;
+        } else {
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                const uint32_t unit = (uint32_t)(((ks * 2 + (mi >> 1)) & 7) ^ l7);
+                uint32_t a0, a1, a2, a3;
+                ldsm_x4(kbase + (ks >> 2) * 2048 + k_tok_off + (unit << 4), a0, a1, a2, a3);
+                if (ks & 1) mma_16816(sb, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+                else mma_16816(sa, a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+            }
+            x0 = (sa[0] + sb[0]) * p.scale_log2, x1 = (sa[1] + sb[1]) * p.scale_log2;
+            x2 = (sa[2] + sb[2]) * p.scale_log2, x3 = (sa[3] + sb[3]) * p.scale_log2;
         }
-        float x0 = (sa[0] + sb[0]) * p.scale_log2, x1 = (sa[1] + sb[1]) * p.scale_log2;
-        float x2 = (sa[2] + sb[2]) * p.scale_log2, x3 = (sa[3] + sb[3]) * p.scale_log2;
         if (row >= nvalid) x0 = x1 = -INFINITY;
         if (row + 8 >= nvalid) x2 = x3 = -INFINITY;
 
@@ -441,23 +504,52 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
         const float p2 = fast_exp2(x2 - mn0), p3 = fast_exp2(x3 - mn1);
         // the row sum uses the bf16-rounded weights that PV multiplies, so that the
         // normalised output is an exact convex mix of V rows
-        const uint32_t pk0 = pack_bf16(p0, p1), pk1 = pack_bf16(p2, p3);
-        l0 = l0 * al0 + bf16_lo(pk0) + bf16_lo(pk1);
-        l1 = l1 * al1 + bf16_hi(pk0) + bf16_hi(pk1);
+        uint32_t pk0, pk1;
+        if constexpr (FP8) {
+            // each key's V scale rides on its weight into the MMA; the row sum is over the weights themselves
+            pk0 = pack_f16(p0 * sv_lo, p1 * sv_lo), pk1 = pack_f16(p2 * sv_hi, p3 * sv_hi);
+            l0 = l0 * al0 + p0 + p2;
+            l1 = l1 * al1 + p1 + p3;
+        } else {
+            pk0 = pack_bf16(p0, p1), pk1 = pack_bf16(p2, p3);
+            l0 = l0 * al0 + bf16_lo(pk0) + bf16_lo(pk1);
+            l1 = l1 * al1 + bf16_hi(pk0) + bf16_hi(pk1);
+        }
         const uint32_t pb0 = movmatrix_t(pk0);
         const uint32_t pb1 = movmatrix_t(pk1);
 
         // O^T += V^T P^T : d x 8 head columns
+        if constexpr (FP8) {
+            // A transposed ldmatrix over 16-bit units hands the thread, per 16-byte chunk u, the bytes
+            // V[token 2c][d], V[token 2c][d + 1], V[token 2c + 1][d], V[token 2c + 1][d + 1] with d = 16 u + 2 row
+            // (tokens 2c, 2c + 1 of the first eight in one register, of the second eight in the next); a byte
+            // permute pairs the two tokens of one d, so accumulator row `row` is d and row `row + 8` is d + 1.
 #pragma unroll
-        for (int mt = 0; mt < KS; ++mt) {
-            o[mt][0] *= al0;
-            o[mt][1] *= al1;
-            o[mt][2] *= al0;
-            o[mt][3] *= al1;
-            const uint32_t unit = (uint32_t)(((mt * 2 + (mi & 1)) & 7) ^ l7);
-            uint32_t a0, a1, a2, a3;
-            ldsm_x4_t(vbase + (mt >> 2) * 2048 + v_tok_off + (unit << 4), a0, a1, a2, a3);
-            mma_16816(o[mt], a0, a1, a2, a3, pb0, pb1);
+            for (int mp = 0; mp < KS / 2; ++mp) {
+                o[2 * mp][0] *= al0, o[2 * mp][1] *= al1, o[2 * mp][2] *= al0, o[2 * mp][3] *= al1;
+                o[2 * mp + 1][0] *= al0, o[2 * mp + 1][1] *= al1, o[2 * mp + 1][2] *= al0, o[2 * mp + 1][3] *= al1;
+                const uint32_t unit = (uint32_t)(((mp * 2 + (mi >> 1)) & 7) ^ l7);
+                uint32_t r0, r1, r2, r3;
+                ldsm_x4_t(vbase + k_tok_off + (unit << 4), r0, r1, r2, r3);
+                r0 = __byte_perm(r0, 0, 0x3120), r1 = __byte_perm(r1, 0, 0x3120);
+                r2 = __byte_perm(r2, 0, 0x3120), r3 = __byte_perm(r3, 0, 0x3120);
+                mma_16816_f16(o[2 * mp], e4m3x2_to_f16x2(r0), e4m3x2_to_f16x2(r0 >> 16), e4m3x2_to_f16x2(r1), e4m3x2_to_f16x2(r1 >> 16),
+                              pb0, pb1);
+                mma_16816_f16(o[2 * mp + 1], e4m3x2_to_f16x2(r2), e4m3x2_to_f16x2(r2 >> 16), e4m3x2_to_f16x2(r3), e4m3x2_to_f16x2(r3 >> 16),
+                              pb0, pb1);
+            }
+        } else {
+#pragma unroll
+            for (int mt = 0; mt < KS; ++mt) {
+                o[mt][0] *= al0;
+                o[mt][1] *= al1;
+                o[mt][2] *= al0;
+                o[mt][3] *= al1;
+                const uint32_t unit = (uint32_t)(((mt * 2 + (mi & 1)) & 7) ^ l7);
+                uint32_t a0, a1, a2, a3;
+                ldsm_x4_t(vbase + (mt >> 2) * 2048 + v_tok_off + (unit << 4), a0, a1, a2, a3);
+                mma_16816(o[mt], a0, a1, a2, a3, pb0, pb1);
+            }
         }
 
         __syncwarp();  // every lane has read this stage
@@ -480,12 +572,12 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_kernel(const DecodePara
 
 int decode_warps_per_sm() { return kWarps; }
 
-template <int D>
+template <int D, bool FP8>
 static ps_status launch_decode_d(const RunArgs& a) {
-    using Cfg = DecodeCfg<D>;
+    using Cfg = DecodeCfg<D, FP8>;
     static PerDeviceOnce configured;
     const ps_status cfg = once_per_device(configured, []() -> ps_status {
-        PS_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+        PS_CUDA_TRY(cudaFuncSetAttribute(decode_kernel<D, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
         return PS_OK;
     });
     if (cfg != PS_OK) return cfg;
@@ -516,14 +608,15 @@ static ps_status launch_decode_d(const RunArgs& a) {
     p.wait_limit_ns = a.wait_limit_ns;
     int grid = (a.w.n_units + kWarps - 1) / kWarps;
     if (grid > a.dec_sms) grid = a.dec_sms;
-    decode_kernel<D><<<grid, kWarps * 32, Cfg::kSmemBytes, a.stream>>>(p);
+    decode_kernel<D, FP8><<<grid, kWarps * 32, Cfg::kSmemBytes, a.stream>>>(p);
     PS_CUDA_TRY(cudaGetLastError());
     return PS_OK;
 }
 
 ps_status launch_decode(const RunArgs& a) {
     if (a.w.n_units == 0) return PS_OK;
-    return a.shape.head_dim == 128 ? launch_decode_d<128>(a) : launch_decode_d<64>(a);
+    if (a.shape.dtype == 1) return launch_decode_d<128, true>(a);  // the FP8 cache variant exists for head_dim 128
+    return a.shape.head_dim == 128 ? launch_decode_d<128, false>(a) : launch_decode_d<64, false>(a);
 }
 
 }  // namespace ps

@@ -29,7 +29,8 @@ ps_status check_shape(const ps_shape* s) {
     if (s->head_dim != 64 && s->head_dim != 128)
         return fail(PS_ERR_UNSUPPORTED, "head_dim=%d: only 64 and 128 are supported", s->head_dim);
     if (s->page_size != kPage) return fail(PS_ERR_UNSUPPORTED, "page_size=%d: only 16 is supported", s->page_size);
-    if (s->dtype != 0) return fail(PS_ERR_UNSUPPORTED, "dtype=%d: only 0 (bf16) is supported", s->dtype);
+    if (s->dtype != 0 && s->dtype != 1) return fail(PS_ERR_UNSUPPORTED, "dtype=%d: 0 (bf16 cache) and 1 (FP8 E4M3 cache) are supported", s->dtype);
+    if (s->dtype == 1 && s->head_dim != 128) return fail(PS_ERR_UNSUPPORTED, "the FP8 cache is supported for head_dim 128 only");
     int G = s->n_q_heads / s->n_kv_heads;
     if (G > 8 || (G & (G - 1)) != 0)
         return fail(PS_ERR_UNSUPPORTED, "q heads per kv head = %d: supported group sizes are 1, 2, 4, 8", G);
@@ -87,6 +88,87 @@ __global__ void kv_gather_kernel(const char* pool, int64_t num_pages, const int3
     }
 }
 
+// ---------------------------------------------------------------------------
+// FP8 (E4M3) cache variant.  Each (token, kv head) vector of K and of V is stored as head_dim E4M3 codes with one
+// fp32 scale: scale = amax / 448 rounded up to 8 significant bits (1 if the vector is zero), code =
+// round-to-nearest-even(x / scale) saturating at +-448, both divisions IEEE fp32.  A token's codes never change
+// when later tokens are appended.  (With 8 significant bits a softmax weight of exactly 1 times the scale is still
+// exact in the 16-bit operand of the decode kernel's MMA.)
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t quantise4(float x0, float x1, float x2, float x3, float scale) {
+    uint16_t lo, hi;  // cvt packs its first operand into the upper byte
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(__fdiv_rn(x1, scale)), "f"(__fdiv_rn(x0, scale)));
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(__fdiv_rn(x3, scale)), "f"(__fdiv_rn(x2, scale)));
+    return (uint32_t)lo | ((uint32_t)hi << 16);
+}
+
+// One warp quantises K and V of one (new token, kv head): lane l holds elements 4 l .. 4 l + 3 (head_dim = 128).
+__global__ void kv_write_fp8_kernel(char* pool, int64_t num_pages, const uint2* __restrict__ k_new,
+                                    const uint2* __restrict__ v_new, const int32_t* __restrict__ block_table, int max_pages,
+                                    const int32_t* __restrict__ q_start, const int32_t* __restrict__ prior, int n, int Hkv,
+                                    int* flag) {
+    constexpr int d = 128;
+    const int lane = threadIdx.x & 31;
+    const int64_t total = (int64_t)q_start[n] * Hkv;
+    for (int64_t vec = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); vec < total;
+         vec += (int64_t)gridDim.x * (blockDim.x >> 5)) {
+        const int t = (int)(vec / Hkv), g = (int)(vec % Hkv);
+        int lo = 0, hi = n - 1;
+        while (lo < hi) {
+            int mid = (lo + hi + 1) >> 1;
+            if (q_start[mid] <= t) lo = mid; else hi = mid - 1;
+        }
+        const int r = lo;
+        const int pos = prior[r] + (t - q_start[r]);
+        const int64_t page = block_table[(int64_t)r * max_pages + pos / kPage];
+        if (page < 0 || page >= num_pages) {
+            if (lane == 0) atomicOr(flag, kStatusBounds);
+            continue;
+        }
+        const int slot = pos % kPage;
+        char* blk = pool + (page * Hkv + g) * fp8_page_head_bytes(d);
+        const uint32_t off = (uint32_t)(slot * d + (((lane >> 2) ^ (slot & 7)) << 4) + 4 * (lane & 3));
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv) {
+            const uint2 w = (kv == 0 ? k_new : v_new)[vec * (d / 4) + lane];
+            const float x0 = bf16_lo(w.x), x1 = bf16_hi(w.x), x2 = bf16_lo(w.y), x3 = bf16_hi(w.y);
+            float amax = fmaxf(fmaxf(fabsf(x0), fabsf(x1)), fmaxf(fabsf(x2), fabsf(x3)));
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+            float scale = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+            uint32_t sbits = __float_as_uint(scale);  // rounded up to 8 significant bits
+            if (sbits & 0xffffu) sbits = (sbits | 0xffffu) + 1u;
+            scale = __uint_as_float(sbits);
+            *reinterpret_cast<uint32_t*>(blk + kv * (kPage * d) + off) = quantise4(x0, x1, x2, x3, scale);
+            if (lane == 0) reinterpret_cast<float*>(blk + 2 * kPage * d)[kv * kPage + slot] = scale;
+        }
+    }
+}
+
+// Codes of logical tokens [0, len) of one sequence, one byte per element, and their scales.
+__global__ void kv_gather_fp8_kernel(const char* pool, int64_t num_pages, const int32_t* __restrict__ bt_row, int len, int Hkv,
+                                     uint32_t* k_out, uint32_t* v_out, float* k_scale_out, float* v_scale_out, int* flag) {
+    constexpr int d = 128;
+    const int64_t total = (int64_t)len * Hkv * (d / 4);
+    for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (int64_t)gridDim.x * blockDim.x) {
+        const int pos = (int)(idx / (Hkv * (d / 4)));
+        const int rem = (int)(idx % (Hkv * (d / 4)));
+        const int g = rem / (d / 4), w = rem % (d / 4);  // 4-byte word of the vector
+        const int64_t page = bt_row[pos / kPage];
+        if (page < 0 || page >= num_pages) { atomicOr(flag, kStatusBounds); continue; }
+        const int slot = pos % kPage;
+        const char* blk = pool + (page * Hkv + g) * fp8_page_head_bytes(d);
+        const uint32_t off = (uint32_t)(slot * d + (((w >> 2) ^ (slot & 7)) << 4) + 4 * (w & 3));
+        if (k_out) k_out[idx] = *reinterpret_cast<const uint32_t*>(blk + off);
+        if (v_out) v_out[idx] = *reinterpret_cast<const uint32_t*>(blk + kPage * d + off);
+        if (w == 0) {
+            const float* sc = reinterpret_cast<const float*>(blk + 2 * kPage * d);
+            if (k_scale_out) k_scale_out[(int64_t)pos * Hkv + g] = sc[slot];
+            if (v_scale_out) v_scale_out[(int64_t)pos * Hkv + g] = sc[kPage + slot];
+        }
+    }
+}
+
 }  // namespace ps
 
 using namespace ps;
@@ -104,7 +186,8 @@ ps_status ps_kv_bytes(const ps_shape* shape, int64_t num_pages, size_t* bytes_ou
     ps_status st = check_shape(shape);
     if (st != PS_OK) return st;
     if (num_pages < 1 || !bytes_out) return fail(PS_ERR_INVALID, "num_pages=%lld or bytes_out invalid", (long long)num_pages);
-    *bytes_out = (size_t)num_pages * shape->n_kv_heads * page_head_bytes(shape->head_dim);
+    *bytes_out = (size_t)num_pages * shape->n_kv_heads *
+                 (shape->dtype == 1 ? fp8_page_head_bytes(shape->head_dim) : page_head_bytes(shape->head_dim));
     return PS_OK;
 }
 
@@ -183,6 +266,15 @@ ps_status ps_kv_write(ps_kv* kv, const void* k_new_dev, const void* v_new_dev, c
     // pool must be stream-ordered because they share meta_dev
     PS_CUDA_TRY(cudaMemcpyAsync(kv->p.meta_dev, meta.data(), meta.size() * sizeof(int32_t), cudaMemcpyHostToDevice, s));
     const int Hkv = kv->p.shape.n_kv_heads, d = kv->p.shape.head_dim;
+    if (kv->p.shape.dtype == 1) {
+        const int64_t warps = T * Hkv;
+        const int blocks = (int)((warps + 7) / 8 < 148 * 16 ? (warps + 7) / 8 : 148 * 16);
+        kv_write_fp8_kernel<<<blocks, 256, 0, s>>>(kv->p.base, kv->p.num_pages, (const uint2*)k_new_dev, (const uint2*)v_new_dev,
+                                                   block_table_dev, max_pages, kv->p.meta_dev, kv->p.meta_dev + n + 1, n, Hkv,
+                                                   kv->p.flag_dev);
+        PS_CUDA_TRY(cudaGetLastError());
+        return PS_OK;
+    }
     const int64_t total = T * Hkv * (d / 8);
     const int threads = 256;
     const int blocks = (int)((total + threads - 1) / threads < 148 * 32 ? (total + threads - 1) / threads : 148 * 32);
@@ -198,6 +290,7 @@ ps_status ps_kv_gather(const ps_kv* kv, const int32_t* block_table_row_dev, int3
     if (!kv || !block_table_row_dev) return fail(PS_ERR_INVALID, "null argument");
     if (len < 0) return fail(PS_ERR_INVALID, "len=%d", len);
     if (len == 0 || (!k_out_dev && !v_out_dev)) return PS_OK;
+    if (kv->p.shape.dtype == 1) return ps_kv_gather_fp8(kv, block_table_row_dev, len, k_out_dev, v_out_dev, nullptr, nullptr, stream);
     const int Hkv = kv->p.shape.n_kv_heads, d = kv->p.shape.head_dim;
     const int64_t total = (int64_t)len * Hkv * (d / 8);
     const int threads = 256;
@@ -205,6 +298,23 @@ ps_status ps_kv_gather(const ps_kv* kv, const int32_t* block_table_row_dev, int3
     kv_gather_kernel<<<blocks, threads, 0, (cudaStream_t)stream>>>(kv->p.base, kv->p.num_pages, block_table_row_dev,
                                                                    len, Hkv, d, (uint4*)k_out_dev, (uint4*)v_out_dev,
                                                                    kv->p.flag_dev);
+    PS_CUDA_TRY(cudaGetLastError());
+    return PS_OK;
+}
+
+ps_status ps_kv_gather_fp8(const ps_kv* kv, const int32_t* block_table_row_dev, int32_t len, void* k_codes_out_dev,
+                           void* v_codes_out_dev, float* k_scale_out_dev, float* v_scale_out_dev, void* stream) {
+    if (!kv || !block_table_row_dev) return fail(PS_ERR_INVALID, "null argument");
+    if (kv->p.shape.dtype != 1) return fail(PS_ERR_INVALID, "the pool does not hold an FP8 cache");
+    if (len < 0) return fail(PS_ERR_INVALID, "len=%d", len);
+    if (len == 0 || (!k_codes_out_dev && !v_codes_out_dev && !k_scale_out_dev && !v_scale_out_dev)) return PS_OK;
+    const int Hkv = kv->p.shape.n_kv_heads;
+    const int64_t total = (int64_t)len * Hkv * 32;
+    const int threads = 256;
+    const int blocks = (int)((total + threads - 1) / threads < 148 * 32 ? (total + threads - 1) / threads : 148 * 32);
+    kv_gather_fp8_kernel<<<blocks, threads, 0, (cudaStream_t)stream>>>(kv->p.base, kv->p.num_pages, block_table_row_dev, len, Hkv,
+                                                                       (uint32_t*)k_codes_out_dev, (uint32_t*)v_codes_out_dev,
+                                                                       k_scale_out_dev, v_scale_out_dev, kv->p.flag_dev);
     PS_CUDA_TRY(cudaGetLastError());
     return PS_OK;
 }

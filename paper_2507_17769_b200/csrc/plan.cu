@@ -452,6 +452,9 @@ ps_status ps_attn_plan(const ps_shape* shape, const int32_t* prior_host, const i
         if ((int64_t)prior_host[r] + q_len_host[r] > (int64_t)max_pages_per_seq * kPage)
             return fail(PS_ERR_INVALID, "request %d: kv_len=%lld exceeds max_pages_per_seq * page_size", r,
                         (long long)prior_host[r] + q_len_host[r]);
+        if (shape->dtype == 1 && q_len_host[r] != 1)
+            return fail(PS_ERR_UNSUPPORTED, "request %d: q_len=%d -- the FP8 cache variant serves decode rows (q_len = 1) only", r,
+                        q_len_host[r]);
         q_start[r] = (int32_t)T;
         T += q_len_host[r];
         if (T > (1 << 24)) return fail(PS_ERR_INVALID, "more than 2^24 new tokens in one batch");

@@ -120,6 +120,7 @@ extern "C" ps_status ps_profile_grid(const ps_shape* shape, const ps_grid_spec* 
     ps_status st = check_shape(shape);
     if (st != PS_OK) return st;
     if (!spec || !rows || !n_rows_out) return fail(PS_ERR_INVALID, "null argument");
+    if (shape->dtype != 0) return fail(PS_ERR_UNSUPPORTED, "the sweep profiles the bf16 cache only");
     if (!spec->chunk_sizes || !spec->decode_counts || !spec->mean_ctxs || spec->n_chunk_sizes < 1 ||
         spec->n_decode_counts < 1 || spec->n_mean_ctxs < 1 || spec->seeds_per_cell < 1 || spec->warmup < 1 || spec->iters < 1)
         return fail(PS_ERR_INVALID, "empty grid axis, or seeds_per_cell / warmup / iters < 1");

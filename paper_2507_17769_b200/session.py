@@ -19,12 +19,13 @@ class PagedAttention:
     >>> out, lse = pa.run(q, block_table_dev)                   # attention
     """
 
-    def __init__(self, n_q_heads, n_kv_heads, head_dim, num_pages, page_size=16, device="cuda", poison=False):
+    def __init__(self, n_q_heads, n_kv_heads, head_dim, num_pages, page_size=16, device="cuda", poison=False, kv_dtype=0):
+        """``kv_dtype``: 0 = bf16 cache, 1 = FP8 (E4M3) cache with a scale per (token, kv head); see ps_shape."""
         import torch
 
         self.torch = torch
         self.device = torch.device(device)
-        self.shape = B.make_shape(n_q_heads, n_kv_heads, head_dim, page_size)
+        self.shape = B.make_shape(n_q_heads, n_kv_heads, head_dim, page_size, kv_dtype)
         self.num_pages = int(num_pages)
         nbytes = B.ps_kv_bytes(self.shape, self.num_pages)
         # 0xFF bytes are bf16 NaN: any read of a slot nobody wrote shows in the output
@@ -63,9 +64,21 @@ class PagedAttention:
         assert k_new.is_contiguous() and v_new.is_contiguous() and block_table_dev.is_contiguous()
         B.ps_kv_write(self.kv, k_new, v_new, block_table_dev, int(max_pages), prior, q_len, self._stream())
 
-    def gather(self, block_table_row_dev, length):
-        """Logical tokens [0, length) of one sequence as contiguous (K, V) bf16 [length, Hkv, d]."""
+    def gather_fp8(self, block_table_row_dev, length):
+        """FP8 cache: logical tokens [0, length) of one sequence as (K codes, V codes) uint8 [length, Hkv, d] and
+        (K scales, V scales) float32 [length, Hkv]."""
         t = self.torch
+        kc = t.empty((length, self.shape.n_kv_heads, self.shape.head_dim), dtype=t.uint8, device=self.device)
+        vc = t.empty_like(kc)
+        ks = t.empty((length, self.shape.n_kv_heads), dtype=t.float32, device=self.device)
+        vs = t.empty_like(ks)
+        B.ps_kv_gather_fp8(self.kv, block_table_row_dev, int(length), kc, vc, ks, vs, self._stream())
+        return kc, vc, ks, vs
+
+    def gather(self, block_table_row_dev, length):
+        """Logical tokens [0, length) of one sequence as contiguous (K, V) bf16 [length, Hkv, d] (bf16 cache)."""
+        t = self.torch
+        assert self.shape.dtype == 0, "use gather_fp8 on an FP8 cache"
         k = t.empty((length, self.shape.n_kv_heads, self.shape.head_dim), dtype=t.bfloat16, device=self.device)
         v = t.empty_like(k)
         B.ps_kv_gather(self.kv, block_table_row_dev, int(length), k, v, self._stream())

@@ -20,7 +20,7 @@ def opts(num_sms=148, dec=0, pre=0):
 
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "polyserve_attn.h")).read()
-    declared = set(re.findall(r"\b(ps_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(ps_[a-z_0-9]+)\s*\(", header))
     assert declared == set(B.EXPORTS)
     lib = B.load()
     for name in declared:

@@ -8,13 +8,14 @@ class DeviceBatch:
     """Pool filled with the batch's K/V (drawn on the device, scattered with
     ``ps_kv_write``), its block table and packed Q as device tensors."""
 
-    def __init__(self, batch: gen.Batch, poison: bool = True, device="cuda"):
+    def __init__(self, batch: gen.Batch, poison: bool = True, device="cuda", kv_dtype: int = 0):
         import torch
         from paper_2507_17769_b200 import PagedAttention
 
         s = batch.shape
         self.batch = batch
-        self.pa = PagedAttention(s.n_q_heads, s.n_kv_heads, s.head_dim, batch.num_pages, s.page_size, device, poison=poison)
+        self.pa = PagedAttention(s.n_q_heads, s.n_kv_heads, s.head_dim, batch.num_pages, s.page_size, device, poison=poison,
+                                 kv_dtype=kv_dtype)
         self.block_table = torch.from_numpy(batch.block_table).to(device)
         for r in range(batch.n):
             L = int(batch.kv_len[r])
