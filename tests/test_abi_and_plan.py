@@ -238,3 +238,50 @@ def test_mixed_batches_split_the_sms_and_single_class_batches_do_not():
     info = ps.ps_plan_get_info(plan)
     assert info.decode_sms + info.prefill_sms == 148 and info.prefill_sms > info.decode_sms  # prefill-heavy batch
     ps.ps_plan_free(plan)
+
+
+def test_replanning_in_place_keeps_the_work_list_slots_where_they_are():
+    """The two work-list slots of the workspace sit at a stride that only grows: a plan object rebuilt for a smaller
+    batch keeps the stride of the larger one (so runs in flight find their slots), and asks for the same workspace
+    again when the larger batch comes back."""
+    s = ps.make_shape(32, 8, 128)
+    big_prior, small_prior = [3000] * 64, [100] * 4
+    plan, ws_big = ps.ps_attn_plan(s, big_prior, [1] * 64, 256, opts())
+    try:
+        fresh_small, ws_small_fresh = ps.ps_attn_plan(s, small_prior, [1] * 4, 256, opts())
+        ps.ps_plan_free(fresh_small)
+        _, ws_small = ps.ps_attn_plan(s, small_prior, [1] * 4, 256, opts(), plan)
+        assert ws_small_fresh < ws_small <= ws_big
+        _, ws_again = ps.ps_attn_plan(s, big_prior, [1] * 64, 256, opts(), plan)
+        assert ws_again == ws_big
+        info = ps.ps_plan_get_info(plan)
+        assert info.n_decode_items >= 64 * 8
+    finally:
+        ps.ps_plan_free(plan)
+
+
+def test_wait_limit_setter_validates_its_argument():
+    s = ps.make_shape(32, 8, 128)
+    plan, _ = ps.ps_attn_plan(s, [100], [1], 16, opts())
+    try:
+        ps.ps_plan_set_wait_limit(plan, 0)
+        ps.ps_plan_set_wait_limit(plan, 4_000_000_000)
+        for bad in (-1, 4_000_000_001):
+            with pytest.raises(ps.PsError) as e:
+                ps.ps_plan_set_wait_limit(plan, bad)
+            assert e.value.status == B.PS_ERR_INVALID
+    finally:
+        ps.ps_plan_free(plan)
+
+
+def test_fp8_cache_shapes_plan_decode_rows_only():
+    s8 = ps.make_shape(32, 8, 128, 16, 1)
+    assert ps.ps_kv_bytes(s8, 3) == 3 * 8 * (2 * 16 * 128 + 2 * 16 * 4)
+    plan, ws = ps.ps_attn_plan(s8, [500, 40], [1, 1], 64, opts())
+    ps.ps_plan_free(plan)
+    with pytest.raises(ps.PsError) as e:
+        ps.ps_attn_plan(s8, [500, 40], [1, 2], 64, opts())
+    assert e.value.status == B.PS_ERR_UNSUPPORTED
+    with pytest.raises(ps.PsError) as e:
+        ps.ps_kv_bytes(ps.make_shape(8, 8, 64, 16, 1), 3)
+    assert e.value.status == B.PS_ERR_UNSUPPORTED

@@ -28,6 +28,12 @@ def test_grid_rows_keys_and_regenerable_lengths(tmp_path):
                     assert r.kv_tokens == int(b.kv_len.sum()) and r.prefill_prior == int(b.prior[n])
                     assert r.decode_bytes == b.decode_bytes() and abs(r.prefill_flops - b.prefill_flops()) < 1e-3 * b.prefill_flops()
                     assert 0 < r.latency_min_us <= r.latency_us <= r.latency_max_us < 1e5
+                    # the rates are the row's own work over its median latency; the fraction uses the nominal peaks here
+                    sec = r.latency_us * 1e-6
+                    assert abs(r.decode_TBps - r.decode_bytes / sec / 1e12) <= 1e-3 * r.decode_TBps + 1e-6
+                    assert abs(r.prefill_TFLOPs - r.prefill_flops / sec / 1e12) <= 1e-3 * r.prefill_TFLOPs + 1e-6
+                    want = max(r.decode_bytes / 8000e9, r.prefill_flops / 2250e12) / sec
+                    assert abs(r.roofline_frac - want) <= 1e-3 * want and 0 < r.roofline_frac < 1.5
     lines = csv.read_text().strip().splitlines()
     assert lines[0].startswith("component,chunk,n_decode") and len(lines) == 1 + len(rows)
     # more KV tokens at the same decode count never makes the batch faster by much
