@@ -20,7 +20,7 @@ precision); decode(code) * scale is evaluated exactly (fp64 holds the 4 + 24
 significant bits).  The attention arithmetic over the dequantised values stays
 the plain fp64 definition (``attn_oracle.c``).
 
-Pins (tests/test_oracle_pins.py): every code round-trips; the encoder equals a
+Pins (tests/test_oracle_fp8_pins.py): every code round-trips; the encoder equals a
 brute-force nearest-value search with ties to the even code; saturation;
 scale = amax / 448; lossless data gives the bf16 oracle's result.
 """
