@@ -98,6 +98,24 @@ def test_split_kv_and_merge_on_the_fp8_cache(seg):
     assert info.n_merge_rows > 0
 
 
+@pytest.mark.parametrize("case", range(16))
+def test_random_decode_batches_on_the_fp8_cache(case):
+    """Seeded batches of decode rows: group sizes 1 to 8, contexts around page and tile boundaries and long ones,
+    default plans, forced segment sizes (split rows and merges) and plans for fewer SMs."""
+    rng = np.random.default_rng(7300 + case)
+    shape = [gen.Shape(8, 8, 128), gen.Shape(16, 8, 128), gen.SHAPE_8B, gen.SHAPE_LARGE][case % 4]
+    ctx = [int(rng.choice([1, 2, 15, 16, 17, 63, 64, 65, 127, 128, 129, int(rng.integers(1, 700)), int(rng.integers(700, 6000))]))
+           for _ in range(int(rng.integers(1, 24)))]
+    opts = None
+    if case % 3 == 1:
+        opts = ps.ps_plan_opts(int(rng.choice([16, 32, 80])), 0, 0)
+    elif case % 3 == 2:
+        opts = ps.ps_plan_opts(0, 0, int(rng.choice([4, 33, 100])))
+    b = gen.make_batch(shape, 7400 + case, [c - 1 for c in ctx], [1] * len(ctx))
+    db, _, _ = check(b, opts, what="fp8 random case %d" % case)
+    db.pa.close()
+
+
 def test_config1_on_the_fp8_cache():
     check(gen.config1(), what="config1 on the fp8 cache")
 
